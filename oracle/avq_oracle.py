@@ -1,0 +1,296 @@
+"""fp64 CPU oracle for the AVQ-attention forward pass.  TEST INFRASTRUCTURE ONLY.
+
+This file is the yardstick the CUDA library is checked against.  It is plain,
+slow numpy in float64, written from the paper's definitions; it shares no code
+with the CUDA path and must never be imported by the product package.  Only the
+test-suite, the smoke check and the benchmark's CPU-baseline leg may call it.
+
+What each function follows in the paper:
+
+* ``assign_head``      - Sec. 3.2 (VQ assignment, ``a(K_j) = argmin_a ||C_a - K_j||^2``)
+                         and Algorithm 1 (parent argmin, then the children of the
+                         chosen parent scanned upward with a strict ``<``).
+* ``aggregate_head``   - Eq. "aggregates" (``n_a`` counts, ``Vbar_a`` value SUMS) and
+                         the two scatter steps of Algorithm 1.
+* ``importance_block`` - Eq. "vqflashattention" + Eq. "importance" and Algorithm 2's
+                         parent pass, with the non-empty-only maximum of the appendix on
+                         numerical stability.
+* ``top_p``            - "Child spawning": the P most important parents of a query tile.
+* ``forward_block_dense``      - the definition: ordinary softmax attention
+                         (Eq. "standardattention") over the block's effective key set, where
+                         a key is represented by its child codeword if its parent was
+                         selected for that block (and the key moved to a child), else by
+                         its parent codeword ("quantised-key attention", Sec. 3.2).
+* ``forward_block_factorised`` - the O(M N) regrouped form of the same quantity
+                         (Sec. 3.2 regrouping + the post-refinement sum of the appendix
+                         "Correcting Attention Derivation": ``A_p Vbar_stay + sum_c A_c Vbar_c``).
+
+Two child-assignment rules are implemented.  REPLACE (default): every key goes
+to the nearest child of its parent.  PARENT_STAYS (Algorithm 1's masked scatter):
+a key moves to that child only if it is strictly closer than the parent.
+
+Readings taken where the paper is silent: ties go to the lowest index
+everywhere; the logit scale is an explicit argument; the importance denominator
+is the exact parent-pass one; query blocks are contiguous ranges of ``block_q``
+queries inside one (batch, head), the last one may be short.
+
+Pins (tests/test_oracle_*.py): brute-force loops on tiny inputs, closed forms,
+conservation laws, the exact-attention special case checked against
+``torch.nn.functional.scaled_dot_product_attention``, and Algorithm 2 re-derived
+literally (mean-recovered parent logits + correcting attention) on codebooks
+that satisfy the parent = mean(children) constraint.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------- assignment
+def _two_smallest(D: np.ndarray):
+    """Smallest and second smallest entry of every row (second = +inf for one column)."""
+    if D.shape[1] == 1:
+        return D[:, 0].copy(), np.full(D.shape[0], np.inf)
+    part = np.partition(D, 1, axis=1)
+    return part[:, 0], part[:, 1]
+
+
+def _rel_margin(d1: np.ndarray, d2: np.ndarray) -> np.ndarray:
+    """(d2 - d1) / d2 with 0/0 counted as a tie (margin 0) and d2 = inf as margin 1."""
+    out = np.ones_like(d1)
+    fin = np.isfinite(d2)
+    pos = fin & (d2 > 0)
+    out[pos] = (d2[pos] - d1[pos]) / d2[pos]
+    out[fin & ~(d2 > 0)] = 0.0
+    return out
+
+
+def assign_head(K, Cp, Cc, parent_stays: bool = False, chunk: int = 1024):
+    """Nearest parent, then nearest child of that parent, for the keys of one head.
+
+    K [N,d], Cp [M,d], Cc [M,C,d].  Distances are the direct form
+    ``sum_k (K_jk - C_ak)^2`` in float64 (Sec. 3.2; Algorithm 1 parent and child steps).
+
+    Returns a dict:
+      parent_idx [N] int64           - argmin over parents, lowest index on ties
+      child_idx  [N] int64           - argmin over the C children of that parent, lowest
+                                       index on ties; -1 where the key stays with the parent
+                                       (only possible with ``parent_stays``)
+      d_parent, d_child [N]          - the winning squared distances
+      parent_margin, child_margin    - relative gap best vs runner-up, (d2-d1)/d2
+      stay_margin                    - relative gap between child and parent distance
+                                       (only meaningful with ``parent_stays``)
+    """
+    K = np.asarray(K, dtype=F64)
+    Cp = np.asarray(Cp, dtype=F64)
+    Cc = np.asarray(Cc, dtype=F64)
+    N, d = K.shape
+    M, C, _ = Cc.shape
+    parent_idx = np.empty(N, dtype=np.int64)
+    child_idx = np.empty(N, dtype=np.int64)
+    d_parent = np.empty(N)
+    d_child = np.empty(N)
+    parent_margin = np.empty(N)
+    child_margin = np.empty(N)
+    for j0 in range(0, N, chunk):
+        j1 = min(N, j0 + chunk)
+        k = K[j0:j1]
+        diff = k[:, None, :] - Cp[None, :, :]
+        Dp = (diff * diff).sum(axis=2)                       # [n, M]
+        a = np.argmin(Dp, axis=1)                            # first minimum = lowest index
+        d1, d2 = _two_smallest(Dp)
+        parent_idx[j0:j1] = a
+        d_parent[j0:j1] = d1
+        parent_margin[j0:j1] = _rel_margin(d1, d2)
+        diffc = k[:, None, :] - Cc[a]                        # [n, C, d]
+        Dc = (diffc * diffc).sum(axis=2)                     # [n, C]
+        c = np.argmin(Dc, axis=1)
+        e1, e2 = _two_smallest(Dc)
+        child_idx[j0:j1] = c
+        d_child[j0:j1] = e1
+        child_margin[j0:j1] = _rel_margin(e1, e2)
+    hi = np.maximum(d_child, d_parent)
+    stay_margin = np.where(hi > 0, np.abs(d_child - d_parent) / np.where(hi > 0, hi, 1.0), 0.0)
+    if parent_stays:
+        moved = d_child < d_parent                           # strict, Algorithm 1's masked scatter
+        child_idx = np.where(moved, child_idx, -1)
+    return dict(parent_idx=parent_idx, child_idx=child_idx, d_parent=d_parent, d_child=d_child,
+                parent_margin=parent_margin, child_margin=child_margin, stay_margin=stay_margin)
+
+
+# --------------------------------------------------------------------------- aggregation
+def aggregate_head(V, parent_idx, child_idx, M: int, C: int):
+    """Per-codeword value sums and key counts for one head (Eq. "aggregates", Algorithm 1).
+
+    Parents collect every key assigned to them; child (m, c) collects the keys
+    with ``parent_idx == m`` and ``child_idx == c`` (keys with child_idx -1 stay).
+    Returns Vp [M,d], np [M], Vc [M,C,d], nc [M,C] in float64.
+    """
+    V = np.asarray(V, dtype=F64)
+    N, d = V.shape
+    Vp = np.zeros((M, d))
+    n_p = np.zeros(M)
+    Vc = np.zeros((M, C, d))
+    n_c = np.zeros((M, C))
+    np.add.at(Vp, parent_idx, V)
+    np.add.at(n_p, parent_idx, 1.0)
+    moved = child_idx >= 0
+    np.add.at(Vc, (parent_idx[moved], child_idx[moved]), V[moved])
+    np.add.at(n_c, (parent_idx[moved], child_idx[moved]), 1.0)
+    return Vp, n_p, Vc, n_c
+
+
+# --------------------------------------------------------------------------- importance, top-P
+def importance_block(Qb, Cp, n_p, scale: float):
+    """Per-parent importance of one query block (Eq. "importance"; Algorithm 2 parent pass).
+
+    ``s = scale * Qb Cp^T``; the row maximum runs over non-empty parents only;
+    ``A = exp(s - m)`` with empty parents zeroed; ``z_i = sum_j A_ij n_j``;
+    ``w_j = sum_i A_ij n_j / z_i``.  Returns (w [M], s [bq,M], m [bq], z [bq]).
+    """
+    Qb = np.asarray(Qb, dtype=F64)
+    Cp = np.asarray(Cp, dtype=F64)
+    n_p = np.asarray(n_p, dtype=F64)
+    s = scale * (Qb @ Cp.T)
+    live = n_p > 0
+    m = np.max(np.where(live[None, :], s, -np.inf), axis=1)
+    A = np.where(live[None, :], np.exp(s - m[:, None]), 0.0)
+    z = A @ n_p
+    w = ((A * n_p[None, :]) / z[:, None]).sum(axis=0)
+    return w, s, m, z
+
+
+def top_p(w, P: int):
+    """Indices of the P largest importances, lowest index first among equals.
+
+    Returns (selected indices ascending [P], relative margin between the P-th and
+    (P+1)-th importance; 1.0 when P is 0 or M, 0.0 for 0/0).
+    """
+    w = np.asarray(w, dtype=F64)
+    M = w.shape[0]
+    order = np.argsort(-w, kind="stable")
+    sel = np.sort(order[:P])
+    if P <= 0 or P >= M:
+        return sel, 1.0
+    a, b = w[order[P - 1]], w[order[P]]
+    margin = (a - b) / a if a > 0 else 0.0
+    return sel, float(margin)
+
+
+# --------------------------------------------------------------------------- forward, one block
+def effective_keys(Cp, Cc, parent_idx, child_idx, selected):
+    """Codeword that represents each key for a block whose refined parents are ``selected``."""
+    Cp = np.asarray(Cp, dtype=F64)
+    Cc = np.asarray(Cc, dtype=F64)
+    is_sel = np.zeros(Cp.shape[0], dtype=bool)
+    is_sel[np.asarray(selected, dtype=np.int64)] = True
+    use_child = is_sel[parent_idx] & (child_idx >= 0)
+    Khat = Cp[parent_idx].copy()
+    Khat[use_child] = Cc[parent_idx[use_child], child_idx[use_child]]
+    return Khat
+
+
+def forward_block_dense(Qb, V, Cp, Cc, parent_idx, child_idx, selected, scale: float):
+    """Softmax attention of a query block over its effective key set, O(bq * N * d).
+
+    Eq. "standardattention" with K_j replaced by the block's effective codeword of key j.
+    """
+    Qb = np.asarray(Qb, dtype=F64)
+    V = np.asarray(V, dtype=F64)
+    Khat = effective_keys(Cp, Cc, parent_idx, child_idx, selected)
+    s = scale * (Qb @ Khat.T)
+    s -= s.max(axis=1, keepdims=True)
+    E = np.exp(s)
+    return (E @ V) / E.sum(axis=1, keepdims=True)
+
+
+def forward_block_factorised(Qb, Cp, Cc, Vp, n_p, Vc, n_c, selected, scale: float):
+    """The same output through per-codeword aggregates, O(bq * (M + P C) * d).
+
+    Unselected parent p contributes ``e^{s_p} (Vp_p, n_p)``.  A selected parent
+    contributes its stay residual ``e^{s_p} (Vp_p - sum_c Vc_pc, n_p - sum_c n_pc)``
+    plus ``e^{s_pc} (Vc_pc, n_pc)`` for each child.  Empty codewords are skipped.
+    """
+    Qb = np.asarray(Qb, dtype=F64)
+    Cp = np.asarray(Cp, dtype=F64)
+    Cc = np.asarray(Cc, dtype=F64)
+    M, C, d = Cc.shape
+    selected = np.asarray(selected, dtype=np.int64)
+    is_sel = np.zeros(M, dtype=bool)
+    is_sel[selected] = True
+    V_stay = Vp - Vc.sum(axis=1)
+    n_stay = n_p - n_c.sum(axis=1)
+    codes = [Cp[~is_sel], Cp[is_sel], Cc[is_sel].reshape(-1, d)]
+    vals = [Vp[~is_sel], V_stay[is_sel], Vc[is_sel].reshape(-1, d)]
+    cnts = [n_p[~is_sel], n_stay[is_sel], n_c[is_sel].reshape(-1)]
+    codes, vals, cnts = np.concatenate(codes), np.concatenate(vals), np.concatenate(cnts)
+    live = cnts > 0
+    codes, vals, cnts = codes[live], vals[live], cnts[live]
+    s = scale * (Qb @ codes.T)
+    s -= s.max(axis=1, keepdims=True)
+    A = np.exp(s)
+    return (A @ vals) / (A @ cnts)[:, None]
+
+
+# --------------------------------------------------------------------------- forward, one head / all heads
+def forward_head(Q, K, V, Cp, Cc, P: int, block_q: int, scale: float, parent_stays: bool = False,
+                 form: str = "dense", blocks=None, assignment=None):
+    """AVQ-attention forward for one (batch, head).
+
+    Q [Nq,d], K,V [Nk,d], Cp [M,d], Cc [M,C,d].  ``form`` is "dense" (definition) or
+    "factorised".  ``blocks`` optionally restricts the evaluation to some query-block
+    indices (rows of other blocks are left NaN).  ``assignment`` may carry a
+    previously computed ``assign_head`` result for these keys.
+
+    Returns a dict: Y [Nq,d]; selected [nblk,P] (ascending, -1 rows for skipped
+    blocks); importance [nblk,M]; topp_margin [nblk]; plus the assignment dict and
+    the aggregates (Vp, np, Vc, nc).
+    """
+    Q = np.asarray(Q, dtype=F64)
+    V = np.asarray(V, dtype=F64)
+    Cp64 = np.asarray(Cp, dtype=F64)
+    Cc64 = np.asarray(Cc, dtype=F64)
+    Nq, d = Q.shape
+    M, C, _ = Cc64.shape
+    asg = assignment if assignment is not None else assign_head(K, Cp64, Cc64, parent_stays)
+    pidx, cidx = asg["parent_idx"], asg["child_idx"]
+    Vp, n_p, Vc, n_c = aggregate_head(V, pidx, cidx, M, C)
+    nblk = (Nq + block_q - 1) // block_q
+    Y = np.full((Nq, d), np.nan)
+    selected = np.full((nblk, P), -1, dtype=np.int64)
+    importance = np.full((nblk, M), np.nan)
+    margins = np.ones(nblk)
+    todo = range(nblk) if blocks is None else blocks
+    for t in todo:
+        i0, i1 = t * block_q, min(Nq, (t + 1) * block_q)
+        Qb = Q[i0:i1]
+        w, _, _, _ = importance_block(Qb, Cp64, n_p, scale)
+        sel, mg = top_p(w, P)
+        importance[t] = w
+        selected[t] = sel
+        margins[t] = mg
+        if form == "dense":
+            Y[i0:i1] = forward_block_dense(Qb, V, Cp64, Cc64, pidx, cidx, sel, scale)
+        elif form == "factorised":
+            Y[i0:i1] = forward_block_factorised(Qb, Cp64, Cc64, Vp, n_p, Vc, n_c, sel, scale)
+        else:
+            raise ValueError(form)
+    return dict(Y=Y, selected=selected, importance=importance, topp_margin=margins, assignment=asg,
+                Vp=Vp, np=n_p, Vc=Vc, nc=n_c)
+
+
+def forward(Q, K, V, Cp, Cc, P: int, block_q: int, scale: float, parent_stays: bool = False,
+            form: str = "dense"):
+    """All (batch, head) pairs.  Q,K,V [B,H,N,d]; Cp [H,M,d]; Cc [H,M,C,d] (one codebook per head)."""
+    B, H = Q.shape[:2]
+    res = [[forward_head(Q[b, h], K[b, h], V[b, h], Cp[h], Cc[h], P, block_q, scale, parent_stays, form)
+            for h in range(H)] for b in range(B)]
+
+    def stack(key):
+        return np.stack([np.stack([res[b][h][key] for h in range(H)]) for b in range(B)])
+
+    out = {k: stack(k) for k in ("Y", "selected", "importance", "topp_margin", "Vp", "np", "Vc", "nc")}
+    for k in ("parent_idx", "child_idx", "parent_margin", "child_margin", "stay_margin"):
+        out[k] = np.stack([np.stack([res[b][h]["assignment"][k] for h in range(H)]) for b in range(B)])
+    return out
