@@ -1,0 +1,189 @@
+/*
+ * avq_attn.h - C ABI of the AVQ-attention forward library for NVIDIA B200 (sm_100a).
+ *
+ * AVQ-attention ("Adaptive Vector-Quantized Attention") replaces the N keys of an
+ * attention layer by M parent codewords, measures per query tile how much attention
+ * mass each parent receives, and refines the P most important parents with their C
+ * pre-learned child codewords.  This library implements the inference forward pass:
+ *
+ *   avq_assign     nearest parent, then nearest child of that parent, per key
+ *                  (Sec. "Vector-Quantized Attention", a(K_j) = argmin_a ||C_a - K_j||^2;
+ *                   Algorithm 1, parent-assignment and child-assignment steps)
+ *   avq_aggregate  per-codeword value sums and key counts
+ *                  (Eq. "aggregates"; Algorithm 1, the two scatter steps)
+ *   avq_forward    assign + aggregate + the attention pass: parent logits and softmax
+ *                  weights (Eq. "vqflashattention"), per-parent importance
+ *                  (Eq. "importance"), top-P selection and child refinement
+ *                  ("Child spawning", "Child attention", Algorithm 2), with the
+ *                  non-empty-only running maximum of the appendix "Numerical Stability
+ *                  of Online Softmax in VQ-Attention".
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless the argument is documented as host.
+ *     The caller owns every buffer.  The library allocates no device memory and keeps
+ *     no mutable global state; calls on different streams with different workspaces
+ *     may overlap.
+ *   - All tensors are dense, row-major, last index fastest:
+ *       Q  [B, H, Nq, d]     K, V [B, H, Nk, d]     Y [B, H, Nq, d]
+ *       Cp [H, M, d]         parent codebook, one per head, shared over the batch
+ *       Cc [H, M, C, d]      child codebook; children of parent m are rows Cc[h, m, 0..C-1]
+ *     (the paper's single [H, M(1+C), d] buffer is the case Cc = Cp + M*d per head, with
+ *     child (m, c) at flat index M + m*C + c).
+ *   - dtype is the element type of Q, K, V, Cp, Cc and Y: float32 or bfloat16.
+ *     Indices are int32, aggregates and importances float32 (counts are exact integers).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Calls are asynchronous with respect to the host unless stated otherwise.
+ *   - The logit scale is explicit (the paper drops the customary 1/sqrt(d) "for clarity").
+ *   - Ties: the lowest index wins in both argmins and in the top-P selection.
+ *   - Query tiles ("Block_N" of Algorithm 2) are contiguous runs of block_q queries inside
+ *     one (batch, head); the last one may be shorter.  block_q changes the result, since
+ *     each tile selects its own P parents.
+ *
+ * Errors: every entry point validates its arguments on the host and returns a status
+ * without launching anything when they are unusable.  Shapes outside the supported
+ * envelope give AVQ_ERR_UNSUPPORTED; there is no silent fallback.  Device-side waits are
+ * bounded; a kernel that gives up records a code in the workspace header which
+ * avq_check() reports as AVQ_ERR_DEVICE_TIMEOUT.
+ */
+#ifndef AVQ_ATTN_H_
+#define AVQ_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define AVQ_API __attribute__((visibility("default")))
+#else
+#define AVQ_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  AVQ_OK = 0,
+  AVQ_ERR_NULL = 1,           /* a required pointer is NULL                               */
+  AVQ_ERR_SHAPE = 2,          /* a size is non-positive or inconsistent (e.g. P > M)      */
+  AVQ_ERR_UNSUPPORTED = 3,    /* valid problem, but outside what the kernels handle       */
+  AVQ_ERR_ALIGN = 4,          /* a pointer is not 16-byte aligned                          */
+  AVQ_ERR_WORKSPACE = 5,      /* workspace missing or smaller than avq_workspace_bytes()  */
+  AVQ_ERR_CUDA = 6,           /* a CUDA runtime / driver call failed                      */
+  AVQ_ERR_DEVICE_TIMEOUT = 7  /* a bounded device-side wait expired (see avq_check)       */
+} avq_status;
+
+typedef enum { AVQ_F32 = 0, AVQ_BF16 = 1 } avq_dtype;
+
+enum {
+  /* Algorithm 1's masked scatter: a key moves to its nearest child only if that child is
+   * strictly closer than the parent; otherwise it stays with the parent (child index -1).
+   * Default (flag clear): every key is represented by the nearest child of its parent.
+   * Supported by the plain CUDA-core kernels only. */
+  AVQ_FLAG_PARENT_STAYS = 1u,
+  /* Use the plain CUDA-core (FFMA) kernels even where a tensor-core kernel exists.
+   * float32 problems always use them.  Meant for cross-checks and for shapes outside the
+   * tensor-core envelope. */
+  AVQ_FLAG_SIMT = 2u
+};
+
+typedef struct {
+  int32_t B, H;        /* batch, heads                                                   */
+  int32_t Nq, Nk;      /* queries and keys per (batch, head)                             */
+  int32_t d;           /* head dimension                                                 */
+  int32_t M, C;        /* parents per head, children per parent                          */
+  int32_t dtype;       /* avq_dtype of Q, K, V, Cp, Cc, Y                                */
+  float scale;         /* logits are scale * <q, c>                                      */
+  uint32_t flags;      /* AVQ_FLAG_*                                                     */
+} avq_problem;
+
+/* Supported envelope.
+ *   CUDA-core kernels (float32, or AVQ_FLAG_SIMT): d % 4 == 0, 4 <= d <= 256; 1 <= M <= 1024;
+ *     1 <= C <= 16; 0 <= P <= M; 1 <= block_q <= 256; M + P*C <= 8192.
+ *   Tensor-core kernels (bfloat16, no flags): d in {64, 128}; M a multiple of 16, 16..256;
+ *     C in {4, 8}; 0 <= P <= M; block_q = 128; AVQ_FLAG_PARENT_STAYS clear.
+ */
+
+/* Bytes of device scratch avq_forward needs for this problem (0 if the problem is invalid).
+ * The workspace holds a 256-byte header (device status word), the key indices and the
+ * aggregates between the three stages.  Host function, no CUDA calls. */
+AVQ_API size_t avq_workspace_bytes(const avq_problem* prob, int32_t P, int32_t block_q);
+
+/* Stage 1.  parent_idx[b,h,j] = argmin_m ||Cp[h,m] - K[b,h,j]||^2  (int32, [B,H,Nk]);
+ * child_idx[b,h,j] = argmin_c ||Cc[h,parent,c] - K[b,h,j]||^2 in [0,C), or -1 when
+ * AVQ_FLAG_PARENT_STAYS is set and no child is strictly closer than the parent.
+ * Distances that are closer than the kernels' arithmetic can separate are re-evaluated
+ * in float64 in the direct form sum_k (K_k - C_k)^2, so the result equals the exact argmin
+ * with lowest-index tie-break.  Uses Nk, d, M, C, B, H, dtype, flags of `prob`. */
+AVQ_API avq_status avq_assign(const avq_problem* prob, const void* K, const void* Cp, const void* Cc,
+                      int32_t* parent_idx, int32_t* child_idx, void* stream);
+
+/* Stage 2.  Vp[b,h,m,:] = sum of V rows whose parent is m, np_[b,h,m] their number;
+ * Vc[b,h,m,c,:], nc[b,h,m,c] the same over keys with (parent, child) = (m, c); keys with
+ * child index -1 enter the parent sums only.  All four outputs are float32 and are
+ * overwritten (the call zeroes them first).  Summation order is not fixed, so the last
+ * bits of the sums may differ from run to run; counts are exact. */
+AVQ_API avq_status avq_aggregate(const avq_problem* prob, const void* V, const int32_t* parent_idx,
+                         const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc,
+                         void* stream);
+
+/* The whole forward: stages 1 and 2 into the workspace, then per query tile
+ *   s = scale * Q_I Cp^T;  m_i = max over non-empty parents;  A = exp(s - m), 0 for empty;
+ *   z_i = sum_j A_ij n_j;  w_j = sum_{i in I} A_ij n_j / z_i          (importance)
+ *   S = the P parents with largest w (ties -> lower index)
+ *   Y_I = [ sum_{p not in S} A_p Vp_p + sum_{p in S} ( A_p Vstay_p + sum_c A_pc Vc_pc ) ]
+ *         / [ the same with counts ],   Vstay = Vp - sum_c Vc (zero unless PARENT_STAYS),
+ * evaluated with one running maximum over all non-empty columns.
+ *   Y              [B,H,Nq,d], dtype of Q
+ *   topp_out       optional (may be NULL): int32 [B,H,ceil(Nq/block_q),P], ascending indices
+ *   importance_out optional (may be NULL): float32 [B,H,ceil(Nq/block_q),M]
+ *   workspace      device scratch of at least avq_workspace_bytes() bytes, 256-byte aligned;
+ *                  its contents are overwritten; after the call it holds, at the offsets
+ *                  avq_workspace_layout() reports, the indices and aggregates of this call.
+ */
+AVQ_API avq_status avq_forward(const avq_problem* prob, const void* Q, const void* K, const void* V,
+                       const void* Cp, const void* Cc, int32_t P, int32_t block_q, void* Y,
+                       int32_t* topp_out, float* importance_out, void* workspace,
+                       size_t workspace_bytes, void* stream);
+
+/* Stage 3 alone: the attention pass of avq_forward over a workspace that a previous
+ * avq_forward call with the same `prob`, P and block_q (and the same K, V, Cp, Cc) filled.
+ * Reads the aggregates from the workspace, recomputes Y (and the optional outputs) for Q.
+ * Lets a caller reuse one set of keys for several query tensors, and lets a profiler time
+ * the attention kernel by itself.  Arguments as in avq_forward. */
+AVQ_API avq_status avq_attend(const avq_problem* prob, const void* Q, const void* Cp, const void* Cc,
+                      int32_t P, int32_t block_q, void* Y, int32_t* topp_out, float* importance_out,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same computation for callers whose Q, K, V and Y live in HOST memory (pinned memory lets
+ * the copies overlap; pageable memory works but serialises).  dQ, dK, dV, dY are device
+ * staging buffers of the tensors' sizes, supplied by the caller.  The call enqueues
+ * host->device copies of Q, K, V, the forward, and the device->host copy of Y on `stream`
+ * and returns; synchronise the stream before reading hY.  Cp, Cc stay device pointers
+ * (they are model parameters). */
+AVQ_API avq_status avq_forward_host(const avq_problem* prob, const void* hQ, const void* hK, const void* hV,
+                            const void* Cp, const void* Cc, int32_t P, int32_t block_q, void* hY,
+                            void* dQ, void* dK, void* dV, void* dY, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
+/* Byte offsets inside the workspace of what avq_forward leaves there.  Any pointer may be
+ * NULL.  parent/child: int32 [B,H,Nk]; Vp f32 [B,H,M,d]; np f32 [B,H,M]; Vc f32 [B,H,M,C,d];
+ * nc f32 [B,H,M,C].  Host function. */
+AVQ_API avq_status avq_workspace_layout(const avq_problem* prob, int32_t P, int32_t block_q,
+                                size_t* parent_idx_off, size_t* child_idx_off, size_t* Vp_off,
+                                size_t* np_off, size_t* Vc_off, size_t* nc_off);
+
+/* Waits for `stream`, reads the status word in the workspace header and clears it.
+ * AVQ_OK, AVQ_ERR_DEVICE_TIMEOUT (a bounded wait inside a kernel expired; outputs of that
+ * call are not valid) or AVQ_ERR_CUDA.  Blocks the host. */
+AVQ_API avq_status avq_check(void* workspace, void* stream);
+
+/* Static, NUL-terminated description of a status code. */
+AVQ_API const char* avq_status_string(avq_status s);
+
+/* Library version as major*10000 + minor*100 + patch. */
+AVQ_API int32_t avq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AVQ_ATTN_H_ */

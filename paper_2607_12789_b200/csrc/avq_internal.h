@@ -1,0 +1,62 @@
+// Internal declarations shared by the translation units of libavq_attn (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "avq_attn.h"
+
+namespace avq {
+
+// Byte offsets of the regions of an avq_forward workspace.
+struct Layout {
+  size_t header = 0;       // 256 bytes; int32 status word at offset 0
+  size_t parent_idx = 0;   // int32 [B,H,Nk]
+  size_t child_idx = 0;    // int32 [B,H,Nk]
+  size_t Vp = 0;           // f32 [B,H,M,d]
+  size_t np = 0;           // f32 [B,H,M]
+  size_t Vc = 0;           // f32 [B,H,M,C,d]
+  size_t nc = 0;           // f32 [B,H,M,C]
+  size_t VpT = 0;          // bf16 [B,H,d,M]      (tensor-core path only)
+  size_t VcT = 0;          // bf16 [B,H,M,d,C]... see avq_tc_finalize (tensor-core path only)
+  size_t total = 0;
+};
+
+// Device status codes written to the workspace header by kernels that give up on a wait.
+enum DeviceCode : int32_t {
+  DEV_OK = 0,
+  DEV_TIMEOUT_ASSIGN = 101,
+  DEV_TIMEOUT_ATTEND = 102,
+};
+
+bool use_tensor_path(const avq_problem& p);
+avq_status validate_problem(const avq_problem* p);
+avq_status validate_forward(const avq_problem* p, int32_t P, int32_t block_q);
+Layout make_layout(const avq_problem& p, int32_t P, int32_t block_q);
+
+// ---- plain CUDA-core kernels (avq_simt.cu) ----
+avq_status simt_assign(const avq_problem& p, const void* K, const void* Cp, const void* Cc,
+                       int32_t* parent_idx, int32_t* child_idx, cudaStream_t st);
+avq_status simt_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
+                          const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc,
+                          cudaStream_t st);
+avq_status simt_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc,
+                       const float* Vp, const float* np_, const float* Vc, const float* nc, int32_t P,
+                       int32_t block_q, void* Y, int32_t* topp_out, float* importance_out,
+                       cudaStream_t st);
+
+// ---- tensor-core kernels (avq_tc_*.cu) ----
+avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const void* Cc,
+                     int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, cudaStream_t st);
+avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
+                        const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc,
+                        void* VpT, void* VcT, cudaStream_t st);
+avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc,
+                     const float* np_, const float* nc, const void* VpT, const void* VcT, int32_t P,
+                     void* Y, int32_t* topp_out, float* importance_out, int32_t* status_word,
+                     cudaStream_t st);
+
+inline avq_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? AVQ_OK : AVQ_ERR_CUDA; }
+
+}  // namespace avq

@@ -1,0 +1,97 @@
+"""Shared helpers for the GPU parity tests: run the CUDA library on a seeded workload and
+compare every stage boundary with the fp64 oracle, element by element."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import avq_oracle as orc
+from paper_2607_12789_b200 import binding, synth
+
+NEAR_TIE = 1e-6          # relative margin below which an index / selection flip is excused (and counted)
+TOL = {"f32": dict(max_abs=1e-4, rel_l2=None), "bf16": dict(max_abs=2e-2, rel_l2=5e-3)}
+
+
+def to_device(x: dict, dtype: str) -> dict:
+    td = torch.float32 if dtype == "f32" else torch.bfloat16
+    return {k: torch.from_numpy(v).to("cuda").to(td).contiguous() for k, v in x.items()}
+
+
+def gpu_forward(wl: synth.Workload, x: dict, flags: int = 0, P: int | None = None):
+    dv = to_device(x, wl.dtype)
+    P = wl.P if P is None else P
+    Y, topp, imp, inter = binding.forward(dv["Q"], dv["K"], dv["V"], dv["Cp"], dv["Cc"], P, wl.block_q,
+                                          scale=wl.scale, flags=flags, aux=True)
+    torch.cuda.synchronize()
+    out = dict(Y=Y.float().cpu().numpy().astype(np.float64), selected=topp.cpu().numpy(),
+               importance=imp.cpu().numpy())
+    out.update({k: v.cpu().numpy() for k, v in inter.items()})
+    return out
+
+
+def compare_indices(gpu, ref):
+    """Bit-exact indices except where the oracle's own margin is a near-tie.  Returns counters."""
+    pm = gpu["parent_idx"] != ref["parent_idx"]
+    p_excused = pm & (ref["parent_margin"] < NEAR_TIE)
+    assert not (pm & ~p_excused).any(), f"{(pm & ~p_excused).sum()} parent mismatches outside near-ties"
+    cm = (gpu["child_idx"] != ref["child_idx"]) & ~pm
+    c_excused = cm & ((ref["child_margin"] < NEAR_TIE) | (ref["stay_margin"] < NEAR_TIE))
+    assert not (cm & ~c_excused).any(), f"{(cm & ~c_excused).sum()} child mismatches outside near-ties"
+    return dict(parent_flips_excused=int(p_excused.sum()), child_flips_excused=int(c_excused.sum()),
+                parent_near_ties=int((ref["parent_margin"] < NEAR_TIE).sum()),
+                child_near_ties=int((ref["child_margin"] < NEAR_TIE).sum()))
+
+
+def compare_aggregates(gpu, ref, atol=2e-3):
+    for k in ("np", "nc"):
+        assert np.array_equal(gpu[k], ref[k]), k
+    for k in ("Vp", "Vc"):
+        err = np.abs(gpu[k] - ref[k]).max()
+        assert err <= atol, (k, err)
+
+
+def compare_selection(gpu, ref):
+    """Top-P sets equal per block except where the P-th / (P+1)-th margin is a near-tie."""
+    sel_g, sel_r = gpu["selected"], ref["selected"]
+    assert sel_g.shape == sel_r.shape
+    same = (sel_g == sel_r).all(axis=-1) if sel_g.shape[-1] else np.ones(sel_g.shape[:-1], bool)
+    excused = ~same & (ref["topp_margin"] < NEAR_TIE)
+    assert not (~same & ~excused).any(), f"{(~same & ~excused).sum()} blocks with a wrong top-P set"
+    if sel_g.shape[-1] > 1:
+        assert (np.diff(sel_g, axis=-1) > 0).all(), "top-P indices must be ascending"
+    imp_ok = np.isclose(gpu["importance"], ref["importance"], rtol=2e-3, atol=2e-4)
+    assert imp_ok.all(), np.abs(gpu["importance"] - ref["importance"]).max()
+    return same, int(excused.sum())
+
+
+def compare_output(Yg, Yr, dtype, row_mask=None):
+    tol = TOL[dtype]
+    if row_mask is not None:
+        Yg, Yr = Yg[row_mask], Yr[row_mask]
+    assert np.isfinite(Yg).all()
+    max_abs = float(np.abs(Yg - Yr).max())
+    rel_l2 = float(np.linalg.norm(Yg - Yr) / np.linalg.norm(Yr))
+    assert max_abs <= tol["max_abs"], f"max-abs {max_abs:.3e} > {tol['max_abs']}"
+    if tol["rel_l2"] is not None:
+        assert rel_l2 <= tol["rel_l2"], f"rel-L2 {rel_l2:.3e} > {tol['rel_l2']}"
+    return max_abs, rel_l2
+
+
+def full_parity(wl: synth.Workload, flags: int = 0, P: int | None = None, parent_stays: bool = False, x=None):
+    """Whole-tensor comparison of every stage; for sizes the oracle finishes in seconds."""
+    x = synth.generate(wl) if x is None else x
+    P = wl.P if P is None else P
+    gpu = gpu_forward(wl, x, flags=flags, P=P)
+    ref = orc.forward(x["Q"], x["K"], x["V"], x["Cp"], x["Cc"], P, wl.block_q, wl.scale,
+                      parent_stays=parent_stays, form="dense")
+    rep = compare_indices(gpu, ref)
+    if rep["parent_flips_excused"] == 0 and rep["child_flips_excused"] == 0:
+        compare_aggregates(gpu, ref)
+    same, excused = compare_selection(gpu, ref)
+    rep["topp_flips_excused"] = excused
+    nq = x["Q"].shape[2]
+    rows_ok = np.repeat(same, wl.block_q, axis=-1)[..., :nq]
+    rep["max_abs"], rep["rel_l2"] = compare_output(gpu["Y"], ref["Y"], wl.dtype, rows_ok)
+    rep["stay_count"] = int((ref["child_idx"] < 0).sum())
+    rep["empty_parents"] = int((ref["np"] == 0).sum())
+    return rep
