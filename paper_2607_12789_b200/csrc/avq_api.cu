@@ -29,7 +29,7 @@ avq_status validate_problem(const avq_problem* p) {
   if (use_tensor_path(*p)) {
     if (p->flags & AVQ_FLAG_PARENT_STAYS) return AVQ_ERR_UNSUPPORTED;
     if (p->d != 64 && p->d != 128) return AVQ_ERR_UNSUPPORTED;
-    if (p->M % 16 != 0 || p->M < 16 || p->M > 256) return AVQ_ERR_UNSUPPORTED;
+    if (p->M % 32 != 0 || p->M < 32 || p->M > 256) return AVQ_ERR_UNSUPPORTED;
     if (p->C != 4 && p->C != 8) return AVQ_ERR_UNSUPPORTED;
   } else {
     if (p->d % 4 != 0 || p->d < 4 || p->d > 256) return AVQ_ERR_UNSUPPORTED;

@@ -19,7 +19,7 @@ struct Layout {
   size_t Vc = 0;           // f32 [B,H,M,C,d]
   size_t nc = 0;           // f32 [B,H,M,C]
   size_t VpT = 0;          // bf16 [B,H,d,M]      (tensor-core path only)
-  size_t VcT = 0;          // bf16 [B,H,M,d,C]... see avq_tc_finalize (tensor-core path only)
+  size_t VcT = 0;          // bf16 [B,H,M,d,C]    (tensor-core path only)
   size_t total = 0;
 };
 

@@ -95,3 +95,46 @@ def full_parity(wl: synth.Workload, flags: int = 0, P: int | None = None, parent
     rep["stay_count"] = int((ref["child_idx"] < 0).sum())
     rep["empty_parents"] = int((ref["np"] == 0).sum())
     return rep
+
+
+def sampled_parity(wl: synth.Workload, heads, blocks_per_head: int = 8, flags: int = 0, seed: int = 0):
+    """Full-size run on the GPU, oracle on a sample: whole heads for assignment and aggregates,
+    a few query blocks per sampled head for importance, selection and output."""
+    x = synth.generate(wl)
+    gpu = gpu_forward(wl, x, flags=flags)
+    g = np.random.default_rng(seed)
+    nblk = (wl.N + wl.block_q - 1) // wl.block_q
+    rep = dict(parent_flips_excused=0, child_flips_excused=0, topp_flips_excused=0, max_abs=0.0, rel_l2=0.0)
+    num = den = 0.0
+    for (b, h) in heads:
+        blocks = sorted(g.choice(nblk, size=min(blocks_per_head, nblk), replace=False).tolist())
+        ref = orc.forward_head(x["Q"][b, h], x["K"][b, h], x["V"][b, h], x["Cp"][h], x["Cc"][h], wl.P, wl.block_q,
+                               wl.scale, form="dense", blocks=blocks)
+        gh = {k: v[b, h] for k, v in gpu.items()}
+        asg = ref["assignment"]
+        r = compare_indices(gh, dict(parent_idx=asg["parent_idx"], child_idx=asg["child_idx"],
+                                     parent_margin=asg["parent_margin"], child_margin=asg["child_margin"],
+                                     stay_margin=asg["stay_margin"]))
+        rep["parent_flips_excused"] += r["parent_flips_excused"]
+        rep["child_flips_excused"] += r["child_flips_excused"]
+        if r["parent_flips_excused"] == 0 and r["child_flips_excused"] == 0:
+            compare_aggregates(gh, ref)
+        sub = dict(selected=gh["selected"][blocks], importance=gh["importance"][blocks])
+        same, excused = compare_selection(sub, dict(selected=ref["selected"][blocks],
+                                                    importance=ref["importance"][blocks],
+                                                    topp_margin=ref["topp_margin"][blocks]))
+        rep["topp_flips_excused"] += excused
+        for t, ok in zip(blocks, same):
+            if not ok:
+                continue
+            rows = slice(t * wl.block_q, min(wl.N, (t + 1) * wl.block_q))
+            yg, yr = gh["Y"][rows], ref["Y"][rows]
+            assert np.isfinite(yg).all()
+            rep["max_abs"] = max(rep["max_abs"], float(np.abs(yg - yr).max()))
+            num += float(((yg - yr) ** 2).sum())
+            den += float((yr ** 2).sum())
+    rep["rel_l2"] = float(np.sqrt(num / den))
+    tol = TOL[wl.dtype]
+    assert rep["max_abs"] <= tol["max_abs"], rep
+    assert tol["rel_l2"] is None or rep["rel_l2"] <= tol["rel_l2"], rep
+    return rep, gpu, x

@@ -1,0 +1,84 @@
+"""GPU parity of the tcgen05 tensor-core path (bf16) against the fp64 oracle.
+
+Small and mid-size configurations are compared whole; the long ones on whole sampled heads
+(assignments, aggregates) and sampled query blocks (importance, top-P, output)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_12789_b200 import binding, synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def test_small_bf16_single_child_tile():
+    rep = parity.full_parity(synth.C1.with_(B=1, H=2, N=512))
+    assert rep["empty_parents"] > 0
+
+
+def test_c1_vitb_full():
+    rep = parity.full_parity(synth.C1)
+    print("c1", rep)
+
+
+def test_c2_mid_full():
+    rep = parity.full_parity(synth.C2)
+    print("c2", rep)
+
+
+def test_c3_long_sampled():
+    rep, gpu, x = parity.sampled_parity(synth.C3, heads=[(0, 3), (0, 12)], blocks_per_head=8)
+    print("c3", rep)
+    # properties that hold at any size, over the whole tensor
+    assert np.isfinite(gpu["Y"]).all()
+    assert np.array_equal(gpu["np"].sum(axis=-1), np.full((1, 16), 16384.0))
+    assert np.array_equal(gpu["nc"].sum(axis=-1), gpu["np"])
+    np.testing.assert_allclose(gpu["importance"].sum(axis=-1), 128.0, rtol=1e-4)
+    np.testing.assert_allclose(gpu["Vp"].sum(axis=2), x["V"].astype(np.float64).sum(axis=2), atol=5e-3)
+
+
+@pytest.mark.parametrize("M", [32, 64, 128, 256])
+def test_sweep_N1024_all_P(M):
+    for P in synth.sweep_P(M):
+        parity.full_parity(synth.sweep_point(1024, M, P).with_(H=4))
+
+
+@pytest.mark.parametrize("M,P", [(64, 16), (256, 64), (128, 128)])
+def test_sweep_N4096(M, P):
+    parity.full_parity(synth.sweep_point(4096, M, P).with_(H=2))
+
+
+def test_sweep_N16384_sampled():
+    parity.sampled_parity(synth.sweep_point(16384, 256, 32), heads=[(0, 5)], blocks_per_head=6)
+
+
+def test_sweep_N65536_sampled():
+    parity.sampled_parity(synth.sweep_point(65536, 64, 16), heads=[(0, 9)], blocks_per_head=4)
+
+
+def test_ragged_tail_and_nq_not_nk():
+    wl = synth.C1.with_(B=1, H=3, N=1000, seed=31)
+    x = synth.generate(wl)
+    x["Q"] = np.ascontiguousarray(x["Q"][:, :, :700])
+    parity.full_parity(wl, x=x)
+
+
+def test_other_shapes_d128_C8_M96():
+    parity.full_parity(synth.Workload("odd", B=1, H=2, N=768, d=128, M=96, C=8, P=12, block_q=128, seed=77,
+                                      alpha=0.5, hot_queries=True))
+
+
+def test_tensor_core_and_cuda_core_paths_agree_at_full_size():
+    wl = synth.C3.with_(H=4)
+    dv = parity.to_device(synth.generate(wl), "bf16")
+    args = (dv["Q"], dv["K"], dv["V"], dv["Cp"], dv["Cc"], wl.P, wl.block_q)
+    Yt, St, Wt, It = binding.forward(*args, scale=wl.scale, aux=True)
+    Ys, Ss, Ws, Is = binding.forward(*args, scale=wl.scale, flags=binding.FLAG_SIMT, aux=True)
+    assert torch.equal(It["parent_idx"], Is["parent_idx"]) and torch.equal(It["child_idx"], Is["child_idx"])
+    assert torch.equal(It["np"], Is["np"]) and torch.equal(It["nc"], Is["nc"])
+    same = (St == Ss).all(dim=-1)
+    assert same.float().mean() > 0.99                      # selections may differ only at near-ties
+    rows = same.repeat_interleave(wl.block_q, dim=-1)
+    diff = (Yt.float() - Ys.float()).abs()[rows]
+    assert diff.max() <= 2e-2
