@@ -165,6 +165,36 @@ AVQ_API avq_status avq_forward_host(const avq_problem* prob, const void* hQ, con
                             void* dQ, void* dK, void* dV, void* dY, void* workspace,
                             size_t workspace_bytes, void* stream);
 
+/* Size of the built-in scratch array avq_forward_static works in. */
+#define AVQ_STATIC_WORKSPACE_BYTES (24u * 1024u * 1024u)
+
+/* avq_forward for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of avq_forward, not a step of the method.)
+ *
+ * Who needs it: code that must not call cudaMalloc where it runs the forward pass - a
+ * plugin given only its input and output buffers, a serving loop whose memory is planned
+ * up front, a real-time path that bans allocator calls after start-up.  avq_forward asks
+ * such callers for a workspace they cannot produce; this entry point uses a fixed
+ * AVQ_STATIC_WORKSPACE_BYTES array inside the library's device image instead, so it makes
+ * no cudaMalloc/cudaFree call and calls no allocating library routine.  Every GPU on which
+ * the library is loaded holds that array until the process exits.
+ *
+ * Arguments and results are those of avq_forward without workspace/workspace_bytes.
+ *   - Problems whose avq_workspace_bytes() exceeds AVQ_STATIC_WORKSPACE_BYTES are rejected
+ *     with AVQ_ERR_WORKSPACE before anything is launched (the three large benchmark
+ *     configurations fit; e.g. B = 4, H = 16, N = 65536 does not).
+ *   - The first call on a device resolves the array's device address (once per device, with
+ *     that device current) and should therefore happen before any stream capture begins.
+ *   - All calls share the one array.  Each call clears what it accumulates into, so calls
+ *     that run one after another are independent; calls that overlap on the GPU (different
+ *     streams, or several host threads) race on it and give wrong results.
+ *   - avq_check_static() is avq_check() on the built-in array. */
+AVQ_API avq_status avq_forward_static(const avq_problem* prob, const void* Q, const void* K, const void* V,
+                              const void* Cp, const void* Cc, int32_t P, int32_t block_q, void* Y,
+                              int32_t* topp_out, float* importance_out, void* stream);
+AVQ_API avq_status avq_check_static(void* stream);
+AVQ_API size_t avq_static_workspace_bytes(void);
+
 /* Byte offsets inside the workspace of what avq_forward leaves there.  Any pointer may be
  * NULL.  parent/child: int32 [B,H,Nk]; Vp f32 [B,H,M,d]; np f32 [B,H,M]; Vc f32 [B,H,M,C,d];
  * nc f32 [B,H,M,C].  Host function. */

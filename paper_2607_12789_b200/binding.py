@@ -21,7 +21,8 @@ STATUS_NAMES = {0: "AVQ_OK", 1: "AVQ_ERR_NULL", 2: "AVQ_ERR_SHAPE", 3: "AVQ_ERR_
                 5: "AVQ_ERR_WORKSPACE", 6: "AVQ_ERR_CUDA", 7: "AVQ_ERR_DEVICE_TIMEOUT"}
 
 EXPORTS = ("avq_workspace_bytes", "avq_assign", "avq_aggregate", "avq_forward", "avq_forward_host", "avq_attend",
-           "avq_workspace_layout", "avq_check", "avq_status_string", "avq_version")
+           "avq_workspace_layout", "avq_check", "avq_status_string", "avq_version", "avq_forward_static",
+           "avq_check_static", "avq_static_workspace_bytes")
 
 
 class AvqProblem(ctypes.Structure):
@@ -63,6 +64,10 @@ def lib() -> ctypes.CDLL:
         L.avq_workspace_layout.restype = i32
         L.avq_workspace_layout.argtypes = [pp, i32, i32, psz, psz, psz, psz, psz, psz]
         L.avq_check.restype, L.avq_check.argtypes = i32, [vp, vp]
+        L.avq_forward_static.restype = i32
+        L.avq_forward_static.argtypes = [pp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
+        L.avq_check_static.restype, L.avq_check_static.argtypes = i32, [vp]
+        L.avq_static_workspace_bytes.restype, L.avq_static_workspace_bytes.argtypes = sz, []
         L.avq_status_string.restype, L.avq_status_string.argtypes = ctypes.c_char_p, [i32]
         L.avq_version.restype, L.avq_version.argtypes = i32, []
         _lib = L
@@ -227,3 +232,24 @@ def forward(Q, K, V, Cp, Cc, P: int, block_q: int, scale=None, flags: int = 0, a
     if aux:
         return Y, f.topp, f.importance, f.intermediates()
     return Y
+
+
+def forward_static(Q, K, V, Cp, Cc, P: int, block_q: int, scale=None, flags: int = 0, aux: bool = False):
+    """avq_forward_static: the forward pass in the library's built-in scratch array, for callers
+    that cannot allocate a workspace.  Only the outputs are torch tensors here; nothing else is
+    allocated on the device.  Returns Y, or (Y, topp, importance) with ``aux``."""
+    _chk(Q, K, V, Cp, Cc)
+    prob = _problem_from(Q, K, Cp, Cc, scale, flags)
+    B, H, Nq, d = Q.shape
+    nblk = (Nq + block_q - 1) // block_q
+    Y = torch.empty_like(Q)
+    topp = torch.empty((B, H, nblk, P), dtype=torch.int32, device=Q.device) if aux else None
+    imp = torch.empty((B, H, nblk, prob.M), dtype=torch.float32, device=Q.device) if aux else None
+    st = lib().avq_forward_static(ctypes.byref(prob), _ptr(Q), _ptr(K), _ptr(V), _ptr(Cp), _ptr(Cc), P, block_q,
+                                  _ptr(Y), _ptr(topp), _ptr(imp), _stream())
+    if st != 0:
+        raise AvqError(st, "avq_forward_static")
+    st = lib().avq_check_static(_stream())
+    if st != 0:
+        raise AvqError(st, "avq_check_static")
+    return (Y, topp, imp) if aux else Y
