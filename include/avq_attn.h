@@ -100,7 +100,7 @@ typedef struct {
  *   CUDA-core kernels (float32, or AVQ_FLAG_SIMT): d % 4 == 0, 4 <= d <= 256; 1 <= M <= 1024;
  *     1 <= C <= 16; 0 <= P <= M; 1 <= block_q <= 256; M + P*C <= 8192.
  *   Tensor-core kernels (bfloat16, no flags): d in {64, 128}; M a multiple of 32, 32..256;
- *     C in {4, 8}; 0 <= P <= M; block_q = 128; AVQ_FLAG_PARENT_STAYS clear.
+ *     C in {4, 8}; 0 <= P <= M; block_q = 128; scale > 0; AVQ_FLAG_PARENT_STAYS clear.
  */
 
 /* Bytes of device scratch avq_forward needs for this problem (0 if the problem is invalid).

@@ -31,6 +31,7 @@ avq_status validate_problem(const avq_problem* p) {
     if (p->d != 64 && p->d != 128) return AVQ_ERR_UNSUPPORTED;
     if (p->M % 32 != 0 || p->M < 32 || p->M > 256) return AVQ_ERR_UNSUPPORTED;
     if (p->C != 4 && p->C != 8) return AVQ_ERR_UNSUPPORTED;
+    if (!(p->scale > 0.f)) return AVQ_ERR_UNSUPPORTED;
   } else {
     if (p->d % 4 != 0 || p->d < 4 || p->d > 256) return AVQ_ERR_UNSUPPORTED;
     if (p->M > 1024 || p->C > 16) return AVQ_ERR_UNSUPPORTED;

@@ -58,9 +58,9 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                  const __nv_bfloat16* __restrict__ Cp, const __nv_bfloat16* __restrict__ Cc,
                  int32_t* __restrict__ pidx, int32_t* __restrict__ cidx, int H, int Nk, int M, int C,
                  uint32_t tmem_cols, int32_t* status_word) {
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>(
-      (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
+  // 1024-byte alignment (swizzle atoms) is requested from the launch, not computed from the pointer, so
+  // that the compiler keeps every access in the shared address space.
+  extern __shared__ __align__(1024) unsigned char smem[];
   constexpr int kSub = D / 64;                       // 64-column sub-tiles along the head dimension
   unsigned char* Ks = smem;                          // kSub x [128 x 128 B]
   unsigned char* Cs = Ks + kSub * kKeys * 128;       // kSub x [M x 128 B]

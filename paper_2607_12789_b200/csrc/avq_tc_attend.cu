@@ -1,20 +1,22 @@
 // Tensor-core attention pass of AVQ-attention (Algorithm 2 in its masked form) for bf16 inputs.
 //
-// One CTA = one query tile of 128 rows of one (batch, head), 8 warps.  The codeword columns are
-// walked as tiles: tile 0 holds the M parents, later tiles hold the children of the selected
-// parents in chunks.  Per tile:
-//   codes [n x d] in shared memory (TMA for parents, gathered rows for children)
-//   S = Q . codes^T          tcgen05.mma, fp32 accumulator in TMEM columns [0, n)
-//   softmax weights          each query row is split over two threads (column halves); the
-//                            row maximum runs over non-empty codewords only; weights of empty
-//                            codewords are zero (appendix on numerical stability)
-//   A (bf16) -> shared       K-major, 128-byte swizzle, in place of the codes
-//   O += A . Vbar            tcgen05.mma into TMEM columns [CT, CT + d)
-// Tile 0 additionally forms the importance w_j = n_j sum_i A_ij / z_i (Eq. "importance") from
-// the fp32 weights, picks the P largest (ties to the lower index) and zeroes the selected
-// parents' columns before they reach the second MMA: their keys are represented by the
-// children instead.  When a later tile raises a row's maximum, that row of O is rescaled in
-// TMEM.  The denominator uses the same bf16-rounded weights as the numerator.
+// One CTA = one query tile of 128 rows of one (batch, head); each row is handled by NQ threads
+// (column slices).  Flow of a tile:
+//   parents   S = Q . Cp^T                 tcgen05.mma, fp32 accumulator in TMEM columns [0, M)
+//             row maximum over non-empty parents, exp2, weights parked in TMEM as fp32,
+//             exact denominator z                                   (Eq. "vqflashattention")
+//             importance w_j = n_j sum_i A_ij / z_i from the fp32 weights  (Eq. "importance")
+//             top-P by rank, ties to the lower index                ("Child spawning")
+//             bf16 weights with the selected parents' columns zeroed -> shared memory
+//             O = A . Vbar_p               tcgen05.mma into TMEM columns [CT, CT + d)
+//   children  of the selected parents, in chunks of <= CHW columns: gathered codeword rows,
+//             S_c = Q . Cc_sel^T, running maximum (non-empty children only), O rescaled in TMEM if a
+//             row's maximum moved, bf16 weights, O += A_c . Vbar_c   (Algorithm 2, child loop)
+//   Y = O / z, z accumulated from the same bf16-rounded weights as the numerator.
+// Empty codewords are excluded from every maximum and contribute nothing (their count and value sum
+// are zero; their weight is clamped so that it stays finite) - appendix on numerical stability.
+// The gathers of the first child chunk are issued early so that their latency hides behind the weight
+// conversion and the parents' second MMA.
 #include "avq_tc_common.cuh"
 
 namespace avq {
@@ -22,8 +24,16 @@ namespace {
 
 using namespace tc;
 
+#ifdef AVQ_PHASE_DEBUG
+// Debug build only: thread 0 of the first CTAs records clock64() at phase boundaries.
+__device__ long long g_phase_clocks[64 * 32];
+#define PHASE_MARK(i) do { if (tid == 0 && blockIdx.x < 8 && blockIdx.y < 8 && (i) < 32) \
+    g_phase_clocks[(blockIdx.y * 8 + blockIdx.x) * 32 + (i)] = clock64(); } while (0)
+#else
+#define PHASE_MARK(i) do { } while (0)
+#endif
+
 constexpr int kRows = 128;
-constexpr int kThreads = 256;
 
 struct AttendParams {
   const __nv_bfloat16* Cc;    // [H, M, C, d]
@@ -35,7 +45,7 @@ struct AttendParams {
   float* importance_out;      // optional
   int32_t* status_word;
   int H, Nq, M, C, P, nblk;
-  int CT;                     // columns per tile (two halves of CT/2), multiple of 32, >= M
+  int logC;                   // log2(C)
   uint32_t tmem_cols;
   float scale_log2e;
 };
@@ -49,7 +59,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-__device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
 // Column sums over the 32 lanes of a warp of V values per lane.  Returns, in every lane, the
 // sum of column (lane >> (5 - log2 V)).  V = 32: 31 shuffles instead of 160.
@@ -76,38 +85,77 @@ __device__ __forceinline__ float transpose_reduce(float (&v)[V], int lane) {
   return v[0];
 }
 
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
+// Rounds 16 fp32 weights to bf16, stores them at (row r, columns col0..col0+15) of the K-major
+// swizzled A tile, and returns sum(rounded weight * count).
+__device__ __forceinline__ float store_weights16(unsigned char* A, int r, int col0, const float* cnt16,
+                                                 const float (&a)[16]) {
+  const float4* n4 = reinterpret_cast<const float4*>(cnt16);
+  uint32_t pk[8];
+  float z = 0.f;
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const float4 n = n4[u];
+    const uint32_t p0 = pack_bf16(a[4 * u], a[4 * u + 1]);
+    const uint32_t p1 = pack_bf16(a[4 * u + 2], a[4 * u + 3]);
+    z = fmaf(__uint_as_float(p0 << 16), n.x, z);
+    z = fmaf(__uint_as_float(p0 & 0xFFFF0000u), n.y, z);
+    z = fmaf(__uint_as_float(p1 << 16), n.z, z);
+    z = fmaf(__uint_as_float(p1 & 0xFFFF0000u), n.w, z);
+    pk[2 * u] = p0;
+    pk[2 * u + 1] = p1;
+  }
+  unsigned char* sub = A + (col0 >> 6) * (kRows * 128);
+  *reinterpret_cast<uint4*>(sub + sw128_offset(r, col0 & 63)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+  *reinterpret_cast<uint4*>(sub + sw128_offset(r, (col0 & 63) + 8)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+  return z;
+}
+
+// NQ = threads per query row: 1, 2 or 4.  Small tiles take NQ = 1 so that four CTAs share an SM and
+// overlap each other's load / MMA / softmax phases; the largest take NQ = 4.
+// CT = parent tile width (64, 128 or 256, >= M), a compile-time constant so that every shared-memory
+// offset folds into the instruction stream instead of occupying a register.
+template <int D, int NQ, int CT>
+__global__ void __launch_bounds__(128 * NQ, 4 / NQ)
 tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmCp,
                  const __grid_constant__ CUtensorMap tmVpT, const AttendParams p) {
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>(
-      (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
+  // 1024-byte alignment (swizzle atoms) is requested from the launch, not computed from the pointer, so
+  // that the compiler keeps every access in the shared address space.
+  extern __shared__ __align__(1024) unsigned char smem[];
+  constexpr int kThreads = 128 * NQ;
   constexpr int kSubD = D / 64;
-  const int CT = p.CT, MH = CT >> 1, M = p.M, C = p.C, P = p.P;
-  const int subA = (CT + 63) >> 6;                       // 64-column sub-tiles of an A / value tile
-  const int ca_bytes = max(CT * D * 2, subA * kRows * 128);
+  constexpr int kLogD = (D == 128) ? 7 : 6;
+  constexpr int kLogChunks = kLogD - 3;                  // 16-byte chunks per codeword row
+  constexpr int CHW = CT < 128 ? CT : 128;               // child chunk width
+  constexpr int QW = CT / NQ, QWC = CHW / NQ;
+  constexpr int subA = CT >> 6;                          // 64-column sub-tiles of an A / value tile
+  constexpr int ca_bytes = (CT * D * 2 > subA * kRows * 128) ? CT * D * 2 : subA * kRows * 128;
+  const int M = p.M, C = p.C, P = p.P, logC = p.logC;
   unsigned char* Qs = smem;                              // kSubD x [128 x 128 B]
-  unsigned char* CA = Qs + kSubD * kRows * 128;          // codes, later the bf16 weights
-  unsigned char* Vs = CA + ca_bytes;                     // subA x [D x 128 B]
-  float* cnt = reinterpret_cast<float*>(Vs + subA * D * 128);   // [CT] counts of the tile's codewords
-  float* w = cnt + CT;                                   // [256] importance
+  unsigned char* CA = Qs + kSubD * kRows * 128;          // parent codes, later the bf16 weights
+  unsigned char* Vs = CA + ca_bytes;                     // subA x [D x 128 B] value sums
+  unsigned char* CC = Vs + subA * D * 128;               // kSubD x [CHW x 128 B] gathered child codes
+  float* cnt = reinterpret_cast<float*>(CC + CHW * D * 2);   // [CT] key counts of the parents
+  float* bias = cnt + CT;                                // [CT] 0 for non-empty parents, -inf for empty
+  float* keep = bias + CT;                               // [CT] 0 for parents selected for refinement, else 1
+  float* cntc = keep + CT;                               // [CHW] key counts of the child chunk
+  float* biasc = cntc + CHW;                             // [CHW]
+  float* w = biasc + CHW;                                // [256] importance
   float* wpart = w + 256;                                // [4][CT]
-  float* xm = wpart + 4 * CT;                            // [2][128] pair exchange: maxima
-  float* xz = xm + 2 * kRows;                            // [2][128] pair exchange: sums
-  float* xz2 = xz + 2 * kRows;                           // [2][128]
-  int* sel_list = reinterpret_cast<int*>(xz2 + 2 * kRows);   // [256]
-  uint32_t* wmask = reinterpret_cast<uint32_t*>(sel_list + 256);   // [8]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(wmask + 8);         // [4]
+  float* xm = wpart + 4 * CT;                            // [4][128] exchange between the threads of a row
+  float* xz = xm + 4 * kRows;                            // [4][128]
+  float* xz2 = xz + 4 * kRows;                           // [4][128]
+  int* sel_list = reinterpret_cast<int*>(xz2 + 4 * kRows);   // [256]
+  uint32_t* wmask = reinterpret_cast<uint32_t*>(sel_list + 256);   // [16]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(wmask + 18);        // [4]  (wmask[16] is a scratch word)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  unsigned char* selS = reinterpret_cast<unsigned char*>(tmem_slot + 2);   // [256]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int q = warp & 3, hf = warp >> 2, r = q * 32 + lane;
+  const int q = warp & 3, cq = warp >> 2, r = q * 32 + lane;
   const int blk = blockIdx.x, bh = blockIdx.y, h = bh % p.H;
   const int i0 = blk * kRows;
   const int rows_valid = min(kRows, p.Nq - i0);
+  const int colbase = cq * QW;
   uint64_t* bar_ld0 = &bars[0];
   uint64_t* bar_ld1 = &bars[1];
   uint64_t* bar_s = &bars[2];
@@ -118,7 +166,9 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (tid == 0) early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
   __syncthreads();
   if (early_exit) return;
+  PHASE_MARK(0);
 
+  // ---- barriers, then the loads first: Q tile + parent codebook, and the parents' value sums
   if (tid == 0) {
     mbar_init(bar_ld0, 1);
     mbar_init(bar_ld1, 1);
@@ -126,26 +176,6 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     mbar_init(bar_pv, 1);
     mbar_fence_init();
     *abort_flag = 0;
-    prefetch_tmap(&tmQ);
-    prefetch_tmap(&tmCp);
-    prefetch_tmap(&tmVpT);
-  }
-  if (warp == 0) {
-    tmem_alloc(tmem_slot, p.tmem_cols);
-    tmem_relinquish();
-  }
-  for (int j = tid; j < CT; j += kThreads) cnt[j] = j < M ? p.np_[(size_t)bh * M + j] : 0.f;
-  selS[tid] = 0;
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  const uint32_t t_s = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(hf * MH);
-  const uint32_t t_o = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(CT + hf * (D / 2));
-  const uint32_t idesc_o = umma_idesc_bf16(kRows, D);
-
-  // ---- stage Q, the parent codebook and the parents' value sums; S = Q . Cp^T
-  if (tid == 0) {
     mbar_expect_tx(bar_ld0, (uint32_t)(kSubD * (kRows + M) * 128));
 #pragma unroll
     for (int s = 0; s < kSubD; ++s) {
@@ -155,6 +185,31 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int subM = (M + 63) >> 6;
     mbar_expect_tx(bar_ld1, (uint32_t)(subM * D * 128));
     for (int s = 0; s < subM; ++s) tma_load_2d(Vs + s * D * 128, &tmVpT, s * 64, bh * D, bar_ld1);
+  }
+  if (warp == 0) {
+    tmem_alloc(tmem_slot, p.tmem_cols);
+    tmem_relinquish();
+  }
+  for (int j = tid; j < CT; j += kThreads) {
+    const float n = j < M ? p.np_[(size_t)bh * M + j] : 0.f;
+    cnt[j] = n;
+    bias[j] = n > 0.f ? 0.f : -INFINITY;
+    keep[j] = 1.f;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+  const uint32_t t_s = t_row + (uint32_t)colbase;
+  const uint32_t t_sc = t_row + (uint32_t)(cq * QWC);
+  const uint32_t t_o = t_row + (uint32_t)(CT + cq * (D / NQ));
+  const uint32_t idesc_o = umma_idesc_bf16(kRows, D);
+  const float sc = p.scale_log2e;
+  PHASE_MARK(1);
+
+  // ---- S = Q . Cp^T
+  if (tid == 0) {
     if (mbar_wait(bar_ld0, 0, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND)) {
       tc_fence_after();
       const uint32_t idesc = umma_idesc_bf16(kRows, M);
@@ -166,253 +221,377 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       umma_commit(bar_s);
     }
   }
-
-  float m_run = -INFINITY, z_run = 0.f;
   uint32_t ph_s = 0, ph_pv = 0;
   const int PC = P * C;
-  int e0 = 0;           // first child column of the current child tile
-  int ncols = M;        // valid columns of the current tile (tile 0: parents)
-  for (int tile = 0;; ++tile) {
-    const int ncols_pad = (ncols + 15) & ~15;
-    const int my_cols = min(max(ncols_pad - hf * MH, 0), MH);   // multiple of 16
+  const int my_cols = min(max(M - colbase, 0), QW);      // multiple of 16 (M % 32 == 0, QW % 16 == 0)
 
-    // ---- wait for S, row maximum over non-empty codewords
-    const bool s_ok = mbar_wait(bar_s, ph_s, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
-    ph_s ^= 1;
-    tc_fence_after();
-    float mloc = -INFINITY;
-    if (s_ok) {
-      for (int c0 = 0; c0 < my_cols; c0 += 16) {
-        float s[16];
-        tmem_ld16(t_s + c0, s);
+  // ---- parents: row maximum over non-empty codewords (empty ones carry a -inf bias)
+  PHASE_MARK(2);
+  mbar_wait(bar_s, ph_s, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+  ph_s ^= 1;
+  tc_fence_after();
+  PHASE_MARK(3);
+  float mx = -INFINITY;
+  for (int c0 = 0; c0 < my_cols; c0 += 16) {
+    float s[16];
+    tmem_ld16(t_s + c0, s);
+    const float4* b4 = reinterpret_cast<const float4*>(bias + colbase + c0);
 #pragma unroll
-        for (int e = 0; e < 16; ++e)
-          if (cnt[hf * MH + c0 + e] > 0.f) mloc = fmaxf(mloc, s[e] * p.scale_log2e);
-      }
+    for (int u = 0; u < 4; ++u) {
+      const float4 b = b4[u];
+      mx = fmaxf(mx, fmaxf(s[4 * u] + b.x, s[4 * u + 1] + b.y));
+      mx = fmaxf(mx, fmaxf(s[4 * u + 2] + b.z, s[4 * u + 3] + b.w));
     }
-    xm[hf * kRows + r] = mloc;
-    __syncthreads();
-    const float m_new = fmaxf(m_run, fmaxf(xm[r], xm[kRows + r]));
-    // m_new is finite from tile 0 on: at least one parent holds a key.
-
-    if (tile == 0) {
-      // ---- fp32 weights back into TMEM, exact denominator of the parent pass
-      float zloc = 0.f;
-      for (int c0 = 0; c0 < my_cols; c0 += 16) {
-        float s[16];
-        tmem_ld16(t_s + c0, s);
+  }
+  xm[cq * kRows + r] = mx * sc;                         // scale > 0: the maximum commutes with it
+  __syncthreads();
+  float m_run = -INFINITY;
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const float n = cnt[hf * MH + c0 + e];
-          s[e] = n > 0.f ? ex2(fmaf(s[e], p.scale_log2e, -m_new)) : 0.f;
-          zloc = fmaf(s[e], n, zloc);
-        }
-        tmem_st16(t_s + c0, s);
+  for (int u = 0; u < NQ; ++u) m_run = fmaxf(m_run, xm[u * kRows + r]);
+  // m_run is finite: at least one parent holds a key.
+  PHASE_MARK(4);
+
+  // ---- fp32 weights parked in TMEM; exact denominator of the parent pass.  Empty parents need no
+  // zeroing: the clamp keeps their weight finite and their count and value sum are zero.
+  {
+    const float negm = -m_run;
+    float zloc = 0.f;
+    for (int c0 = 0; c0 < my_cols; c0 += 16) {
+      float s[16];
+      tmem_ld16(t_s + c0, s);
+      const float4* n4 = reinterpret_cast<const float4*>(cnt + colbase + c0);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float4 n = n4[u];
+        s[4 * u] = ex2(fminf(fmaf(s[4 * u], sc, negm), 0.f));
+        s[4 * u + 1] = ex2(fminf(fmaf(s[4 * u + 1], sc, negm), 0.f));
+        s[4 * u + 2] = ex2(fminf(fmaf(s[4 * u + 2], sc, negm), 0.f));
+        s[4 * u + 3] = ex2(fminf(fmaf(s[4 * u + 3], sc, negm), 0.f));
+        zloc = fmaf(s[4 * u], n.x, zloc);
+        zloc = fmaf(s[4 * u + 1], n.y, zloc);
+        zloc = fmaf(s[4 * u + 2], n.z, zloc);
+        zloc = fmaf(s[4 * u + 3], n.w, zloc);
       }
-      tmem_st_wait();
-      xz[hf * kRows + r] = zloc;
-      __syncthreads();
-      const float zfull = xz[r] + xz[kRows + r];
-      const float inv = (r < rows_valid) ? 1.f / zfull : 0.f;
-      // ---- importance: column sums of A_ij / z_i over the 128 rows
+      tmem_st16(t_s + c0, s);
+    }
+    tmem_st_wait();
+    xz[cq * kRows + r] = zloc;
+  }
+  __syncthreads();
+  PHASE_MARK(5);
+  {
+    float zfull = 0.f;
+#pragma unroll
+    for (int u = 0; u < NQ; ++u) zfull += xz[u * kRows + r];
+    const float inv = (r < rows_valid) ? 1.f / zfull : 0.f;
+    // ---- importance: column sums of A_ij / z_i over the 128 rows (32 per warp, then 4 warps)
+    if ((QW & 31) == 0) {
       for (int c0 = 0; c0 < my_cols; c0 += 32) {
         float v[32];
-        {
-          float a[16];
-          tmem_ld16(t_s + c0, a);
-#pragma unroll
-          for (int e = 0; e < 16; ++e) v[e] = a[e] * inv;
-          if (c0 + 16 < my_cols) {
-            tmem_ld16(t_s + c0 + 16, a);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) v[16 + e] = a[e] * inv;
-          } else {
-#pragma unroll
-            for (int e = 0; e < 16; ++e) v[16 + e] = 0.f;
-          }
-        }
-        const float colsum = transpose_reduce<32>(v, lane);
-        if (c0 + lane < my_cols) wpart[q * CT + hf * MH + c0 + lane] = colsum;
-      }
-      __syncthreads();
-      if (tid < M) {
-        const float wj = cnt[tid] * (wpart[tid] + wpart[CT + tid] + wpart[2 * CT + tid] + wpart[3 * CT + tid]);
-        w[tid] = wj;
-        if (p.importance_out) p.importance_out[((size_t)bh * p.nblk + blk) * M + tid] = wj;
-      }
-      __syncthreads();
-      // ---- top-P by rank, ties to the lower index; ascending list
-      bool mine = false;
-      if (tid < M) {
-        const float wj = w[tid];
-        int rank = 0;
-        for (int k = 0; k < M; ++k) {
-          const float wk = w[k];
-          rank += (wk > wj) || (wk == wj && k < tid);
-        }
-        mine = rank < P;
-        selS[tid] = mine ? 1 : 0;
-      }
-      const uint32_t bal = __ballot_sync(0xffffffffu, mine);
-      if (lane == 0) wmask[warp] = bal;
-      __syncthreads();
-      if (mine) {
-        int pos = __popc(bal & ((1u << lane) - 1u));
-        for (int u = 0; u < warp; ++u) pos += __popc(wmask[u]);
-        sel_list[pos] = tid;
-        if (p.topp_out) p.topp_out[((size_t)bh * p.nblk + blk) * P + pos] = tid;
-      }
-      // ---- masked bf16 weights into shared memory (over the dead codebook), denominator
-      zloc = 0.f;
-      for (int c0 = 0; c0 < my_cols; c0 += 16) {
         float a[16];
         tmem_ld16(t_s + c0, a);
-        uint32_t pk[8];
 #pragma unroll
-        for (int e = 0; e < 16; e += 2) {
-          const int col = hf * MH + c0 + e;
-          const float a0 = selS[col] ? 0.f : bf16_round(a[e]);
-          const float a1 = selS[col + 1] ? 0.f : bf16_round(a[e + 1]);
-          zloc = fmaf(a0, cnt[col], zloc);
-          zloc = fmaf(a1, cnt[col + 1], zloc);
-          pk[e >> 1] = pack_bf16(a0, a1);
-        }
-        const int col0 = hf * MH + c0;
-        unsigned char* sub = CA + (col0 >> 6) * (kRows * 128);
-        *reinterpret_cast<uint4*>(sub + sw128_offset(r, col0 & 63)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-        *reinterpret_cast<uint4*>(sub + sw128_offset(r, (col0 & 63) + 8)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+        for (int e = 0; e < 16; ++e) v[e] = a[e] * inv;
+        tmem_ld16(t_s + c0 + 16, a);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) v[16 + e] = a[e] * inv;
+        const float colsum = transpose_reduce<32>(v, lane);
+        wpart[q * CT + colbase + c0 + lane] = colsum;
       }
-      xz2[hf * kRows + r] = zloc;
-      m_run = m_new;
     } else {
-      // ---- child tile: rescale what has been accumulated if this row's maximum moved
-      const float alpha = ex2(m_run - m_new);
-      if (__any_sync(0xffffffffu, alpha < 1.f)) {
-        for (int c0 = 0; c0 < D / 2; c0 += 16) {
-          float o[16];
-          tmem_ld16(t_o + c0, o);
-#pragma unroll
-          for (int e = 0; e < 16; ++e) o[e] *= alpha;
-          tmem_st16(t_o + c0, o);
-        }
-        tmem_st_wait();
-      }
-      z_run *= alpha;
-      m_run = m_new;
-      float zloc = 0.f;
       for (int c0 = 0; c0 < my_cols; c0 += 16) {
-        float a[16];
-        if (s_ok) tmem_ld16(t_s + c0, a);
-        uint32_t pk[8];
+        float v[16];
+        tmem_ld16(t_s + c0, v);
 #pragma unroll
-        for (int e = 0; e < 16; e += 2) {
-          const int col = hf * MH + c0 + e;
-          const float n0 = cnt[col], n1 = cnt[col + 1];
-          const float a0 = n0 > 0.f ? bf16_round(ex2(fmaf(a[e], p.scale_log2e, -m_new))) : 0.f;
-          const float a1 = n1 > 0.f ? bf16_round(ex2(fmaf(a[e + 1], p.scale_log2e, -m_new))) : 0.f;
-          zloc = fmaf(a0, n0, zloc);
-          zloc = fmaf(a1, n1, zloc);
-          pk[e >> 1] = pack_bf16(a0, a1);
+        for (int e = 0; e < 16; ++e) v[e] *= inv;
+        const float colsum = transpose_reduce<16>(v, lane);
+        if ((lane & 1) == 0) wpart[q * CT + colbase + c0 + (lane >> 1)] = colsum;
+      }
+    }
+  }
+  __syncthreads();
+  PHASE_MARK(6);
+  if (tid < M) {
+    const float wj = cnt[tid] * ((wpart[tid] + wpart[CT + tid]) + (wpart[2 * CT + tid] + wpart[3 * CT + tid]));
+    w[tid] = wj;
+    if (p.importance_out) p.importance_out[((size_t)bh * p.nblk + blk) * M + tid] = wj;
+  }
+  __syncthreads();
+  PHASE_MARK(7);
+
+  // ---- top-P by rank.  Non-negative floats order like their bit patterns, so the comparisons run on
+  // integers.  gt_j = number of strictly larger importances; parent j is selected if gt_j < P, except
+  // that when a group of EQUAL importances straddles the boundary only its lowest indices are kept.
+  // kT threads share one parent's scan.
+  {
+    constexpr int kT = NQ >= 2 ? 2 : 1;                  // 128 * NQ >= kT * M for every launch shape
+    const int j = tid / kT, part = tid % kT;
+    const uint32_t* keys = reinterpret_cast<const uint32_t*>(w);
+    int* gstar = reinterpret_cast<int*>(&wmask[16]);
+    bool mine = false;
+    if (P >= M) {
+      mine = (j < M) && (part == 0);
+    } else if (P > 0) {
+      int gt = 0;
+      if (j < M) {
+        const uint32_t kj = keys[j];
+        const int span = M / kT, kb = part * span;
+#pragma unroll 2
+        for (int k = kb; k < kb + span; k += 4) {
+          const uint4 kk = *reinterpret_cast<const uint4*>(keys + k);
+          asm("{\n\t.reg .pred p0, p1, p2, p3;\n\t"
+              "setp.gt.u32 p0, %1, %5;\n\tsetp.gt.u32 p1, %2, %5;\n\t"
+              "setp.gt.u32 p2, %3, %5;\n\tsetp.gt.u32 p3, %4, %5;\n\t"
+              "@p0 add.s32 %0, %0, 1;\n\t@p1 add.s32 %0, %0, 1;\n\t"
+              "@p2 add.s32 %0, %0, 1;\n\t@p3 add.s32 %0, %0, 1;\n\t}"
+              : "+r"(gt) : "r"(kk.x), "r"(kk.y), "r"(kk.z), "r"(kk.w), "r"(kj));
         }
-        const int col0 = hf * MH + c0;
-        unsigned char* sub = CA + (col0 >> 6) * (kRows * 128);
-        *reinterpret_cast<uint4*>(sub + sw128_offset(r, col0 & 63)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-        *reinterpret_cast<uint4*>(sub + sw128_offset(r, (col0 & 63) + 8)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
       }
-      xz2[hf * kRows + r] = zloc;
+      PHASE_MARK(16);
+      if (kT == 2) gt += __shfl_xor_sync(0xffffffffu, gt, 1);
+      const bool cand = (j < M) && (part == 0) && (gt < P);
+      if (tid == 0) *gstar = 0;
+      const int ncand = __syncthreads_count(cand);
+      PHASE_MARK(17);
+      mine = cand;
+      if (ncand > P) {                                   // uniform: equal importances straddle the boundary
+        if (cand) atomicMax(gstar, gt);                  // the tied group has the largest gt among candidates
+        __syncthreads();
+        const int g = *gstar;
+        const bool tied = cand && gt == g;
+        const uint32_t beq = __ballot_sync(0xffffffffu, tied);
+        if (lane == 0) wmask[warp] = beq;
+        __syncthreads();
+        int epos = __popc(beq & ((1u << lane) - 1u));
+        for (int u = 0; u < warp; ++u) epos += __popc(wmask[u]);
+        mine = cand && (gt < g || epos < P - g);
+        __syncthreads();
+      }
     }
-    fence_proxy_async();
-    tc_fence_before();
+    PHASE_MARK(18);
+    const uint32_t bal = __ballot_sync(0xffffffffu, mine);
+    if (lane == 0) wmask[warp] = bal;
     __syncthreads();
-    z_run += xz2[r] + xz2[kRows + r];
-
-    // ---- O (+)= A . Vbar for this tile
-    if (tid == 0) {
-      tc_fence_after();
-      const bool v_ok = tile > 0 || mbar_wait(bar_ld1, 0, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
-      if (v_ok) {
-        const uint32_t aa = smem_u32(CA), va = smem_u32(Vs);
-        for (int k = 0; k < ncols_pad / 16; ++k)
-          umma_bf16(tmem_base + CT, umma_desc_sw128(aa + (k / 4) * kRows * 128 + (k % 4) * 32),
-                    umma_desc_sw128(va + (k / 4) * D * 128 + (k % 4) * 32), idesc_o, tile > 0 || k > 0);
-      }
-      umma_commit(bar_pv);
+    PHASE_MARK(19);
+    if (mine) {
+      int pos = __popc(bal & ((1u << lane) - 1u));
+      for (int u = 0; u < warp; ++u) pos += __popc(wmask[u]);
+      sel_list[pos] = j;
+      keep[j] = 0.f;
+      if (p.topp_out) p.topp_out[((size_t)bh * p.nblk + blk) * P + pos] = j;
     }
+  }
+  __syncthreads();
+  PHASE_MARK(8);
 
-    // ---- next child tile, if any
-    if (e0 >= PC) break;
-    const int e1 = min(PC, e0 + CT);
-    ncols = e1 - e0;
-    const int np16 = (ncols + 15) & ~15;
-    // The second MMA reads A (in CA) and the values (in Vs): both must be done before they are rewritten.
-    mbar_wait(bar_pv, ph_pv, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
-    ph_pv ^= 1;
+  // ---- first child chunk: start the asynchronous gather of its codeword rows now; it lands while the
+  // weight conversion below runs
+  const __nv_bfloat16* Cch = p.Cc + (size_t)h * M * C * D;
+  const float* ncb = p.nc + (size_t)bh * M * C;
+  int ncols = min(PC, CHW);
+  int np16 = (ncols + 15) & ~15;
+  auto gather_codes = [&](int e_first) {
+    // row e (local column) = Cc[h, sel_list[(e_first+e)/C], (e_first+e)%C, :]; padding rows are zero
+    const int total = np16 << kLogChunks;
+    for (int u = tid; u < total; u += kThreads) {
+      const int row = u >> kLogChunks, ch = u & ((1 << kLogChunks) - 1);
+      unsigned char* dst = CC + (ch >> 3) * (np16 * 128) + sw128_offset(row, (ch & 7) * 8);
+      if (row < ncols) {
+        const int e = e_first + row;
+        cp_async16(dst, Cch + (((size_t)sel_list[e >> logC] << logC) + (e & (C - 1))) * D + ch * 8);
+      } else {
+        *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+      }
+    }
+    if (tid < CHW) {                                     // CHW <= 128 <= kThreads
+      const int e = e_first + tid;
+      const float n = tid < ncols ? ncb[((size_t)sel_list[e >> logC] << logC) + (e & (C - 1))] : 0.f;
+      cntc[tid] = n;
+      biasc[tid] = n > 0.f ? 0.f : -INFINITY;
+    }
+  };
+  gather_codes(0);
+
+  // ---- masked bf16 weights into shared memory (over the dead codebook) + their denominator
+  {
+    float zloc = 0.f;
+    for (int c0 = 0; c0 < my_cols; c0 += 16) {
+      float a[16];
+      tmem_ld16(t_s + c0, a);
+      const float4* k4 = reinterpret_cast<const float4*>(keep + colbase + c0);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float4 kk = k4[u];
+        a[4 * u] *= kk.x;
+        a[4 * u + 1] *= kk.y;
+        a[4 * u + 2] *= kk.z;
+        a[4 * u + 3] *= kk.w;
+      }
+      zloc += store_weights16(CA, r, colbase + c0, cnt + colbase + c0, a);
+    }
+    xz2[cq * kRows + r] = zloc;
+  }
+  cp_async_wait_all();
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  PHASE_MARK(9);
+  float z_run = 0.f;
+#pragma unroll
+  for (int u = 0; u < NQ; ++u) z_run += xz2[u * kRows + r];
+
+  // ---- O = A . Vbar_p, and right behind it the first child chunk's logits
+  if (tid == 0) {
     tc_fence_after();
-    // child codes: row e (local column) = Cc[h, sel_list[(e0+e)/C], (e0+e)%C, :], zero rows as padding
-    {
-      const __nv_bfloat16* Cch = p.Cc + (size_t)h * M * C * D;
-      const int chunks = D / 8;                              // 16-byte chunks per row
-      for (int u = tid; u < np16 * chunks; u += kThreads) {
-        const int row = u / chunks, ch = u % chunks;
-        uint4 val = make_uint4(0, 0, 0, 0);
-        if (row < ncols) {
-          const int e = e0 + row;
-          const int par = sel_list[e / C];
-          val = __ldg(reinterpret_cast<const uint4*>(Cch + ((size_t)par * C + (e % C)) * D) + ch);
-        }
-        unsigned char* sub = CA + (ch >> 3) * (np16 * 128);
-        *reinterpret_cast<uint4*>(sub + sw128_offset(row, (ch & 7) * 8)) = val;
-      }
+    if (mbar_wait(bar_ld1, 0, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND)) {
+      const uint32_t aa = smem_u32(CA), va = smem_u32(Vs);
+      for (int k = 0; k < M / 16; ++k)
+        umma_bf16(tmem_base + CT, umma_desc_sw128(aa + (k / 4) * kRows * 128 + (k % 4) * 32),
+                  umma_desc_sw128(va + (k / 4) * D * 128 + (k % 4) * 32), idesc_o, k > 0);
     }
-    // child values: Vs[k][e] = VcT[bh, par, k, c]; one parent's C children are contiguous per k
-    {
-      const __nv_bfloat16* Vch = p.VcT + (size_t)bh * M * D * C;
-      const int npar = (ncols + C - 1) / C;                  // e0 and ncols are multiples of C
-      const int par0 = e0 / C;
-      for (int u = tid; u < npar * D; u += kThreads) {
-        const int pr = u / D, k = u % D;
-        const int par = sel_list[par0 + pr];
-        const int col = pr * C;
-        unsigned char* dst = Vs + (col >> 6) * (D * 128) + sw128_offset(k, col & 63);
-        const __nv_bfloat16* src = Vch + ((size_t)par * D + k) * C;
-        if (C == 8) *reinterpret_cast<uint4*>(dst) = __ldg(reinterpret_cast<const uint4*>(src));
-        else *reinterpret_cast<uint2*>(dst) = __ldg(reinterpret_cast<const uint2*>(src));
-      }
-      // zero the padding columns [ncols, np16) of the value tile (they meet zero weights, but 0 * NaN is NaN)
-      const int padc = np16 - ncols;
-      for (int u = tid; u < padc * D; u += kThreads) {
-        const int col = ncols + u / D, k = u % D;
-        *reinterpret_cast<__nv_bfloat16*>(Vs + (col >> 6) * (D * 128) + sw128_offset(k, col & 63)) =
-            __float2bfloat16_rn(0.f);
-      }
-      const float* ncb = p.nc + (size_t)bh * M * C;
-      for (int e = tid; e < CT; e += kThreads)
-        cnt[e] = e < ncols ? ncb[(size_t)sel_list[(e0 + e) / C] * C + ((e0 + e) % C)] : 0.f;
-    }
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-    if (tid == 0) {
-      tc_fence_after();
+    umma_commit(bar_pv);
+    if (PC > 0) {
       const uint32_t idesc = umma_idesc_bf16(kRows, np16);
-      const uint32_t qa = smem_u32(Qs), ca = smem_u32(CA);
+      const uint32_t qa = smem_u32(Qs), ca = smem_u32(CC);
 #pragma unroll
       for (int k = 0; k < D / 16; ++k)
         umma_bf16(tmem_base, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
                   umma_desc_sw128(ca + (k / 4) * np16 * 128 + (k % 4) * 32), idesc, k > 0);
       umma_commit(bar_s);
     }
-    e0 = e1;
+  }
+
+  // ---- child chunks
+  const __nv_bfloat16* Vch = p.VcT + (size_t)bh * M * D * C;
+  for (int e0 = 0; e0 < PC; e0 += CHW) {
+    // The previous second MMA must have released A and Vs before they are rewritten.
+    if (e0 == 0) PHASE_MARK(10);
+    mbar_wait(bar_pv, ph_pv, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+    ph_pv ^= 1;
+    tc_fence_after();
+    if (e0 == 0) PHASE_MARK(11);
+    // values of this chunk: Vs[k][e] = VcT[bh, parent, k, child]; one parent's C children are contiguous
+    // per k.  Asynchronous copies: they land while the chunk's logits are turned into weights.
+    {
+      const int npar = ncols >> logC, par0 = e0 >> logC;
+      const int vtotal = npar << kLogD;
+      for (int u = tid; u < vtotal; u += kThreads) {
+        const int pr = u >> kLogD, k = u & (D - 1);
+        const __nv_bfloat16* src = Vch + (((size_t)sel_list[par0 + pr] << kLogD) + k) * C;
+        const int col = pr << logC;
+        unsigned char* dst = Vs + (col >> 6) * (D * 128) + sw128_offset(k, col & 63);
+        if (C == 8) cp_async16(dst, src);
+        else cp_async8(dst, src);
+      }
+    }
+    // zero the padding columns [ncols, np16) of the value tile (they meet finite weights; 0 * NaN is NaN)
+    for (int u = tid; u < ((np16 - ncols) << kLogD); u += kThreads) {
+      const int col = ncols + (u >> kLogD), k = u & (D - 1);
+      *reinterpret_cast<__nv_bfloat16*>(Vs + (col >> 6) * (D * 128) + sw128_offset(k, col & 63)) =
+          __float2bfloat16_rn(0.f);
+    }
+    if (e0 == 0) PHASE_MARK(12);
+
+    // ---- child logits: running maximum over non-empty children
+    mbar_wait(bar_s, ph_s, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+    ph_s ^= 1;
+    tc_fence_after();
+    if (e0 == 0) PHASE_MARK(13);
+    const int my_c = min(max(np16 - cq * QWC, 0), QWC);
+    float mxc = -INFINITY;
+    for (int c0 = 0; c0 < my_c; c0 += 16) {
+      float s[16];
+      tmem_ld16(t_sc + c0, s);
+      const float4* b4 = reinterpret_cast<const float4*>(biasc + cq * QWC + c0);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float4 b = b4[u];
+        mxc = fmaxf(mxc, fmaxf(s[4 * u] + b.x, s[4 * u + 1] + b.y));
+        mxc = fmaxf(mxc, fmaxf(s[4 * u + 2] + b.z, s[4 * u + 3] + b.w));
+      }
+    }
+    xm[cq * kRows + r] = mxc * sc;
+    __syncthreads();
+    float m_new = m_run;
+#pragma unroll
+    for (int u = 0; u < NQ; ++u) m_new = fmaxf(m_new, xm[u * kRows + r]);
+    const float negm = -m_new;
+    if (e0 == 0) PHASE_MARK(14);
+    // ---- rescale what has been accumulated if this row's maximum moved
+    const float alpha = ex2(m_run + negm);
+    if (__any_sync(0xffffffffu, alpha < 1.f)) {
+      for (int c0 = 0; c0 < D / NQ; c0 += 16) {
+        float o[16];
+        tmem_ld16(t_o + c0, o);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) o[e] *= alpha;
+        tmem_st16(t_o + c0, o);
+      }
+      tmem_st_wait();
+    }
+    z_run *= alpha;
+    m_run = m_new;
+    // ---- bf16 weights of the children over the parents' (consumed) weights
+    {
+      float zloc = 0.f;
+      for (int c0 = 0; c0 < my_c; c0 += 16) {
+        float a[16];
+        tmem_ld16(t_sc + c0, a);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) a[e] = ex2(fminf(fmaf(a[e], sc, negm), 0.f));
+        zloc += store_weights16(CA, r, cq * QWC + c0, cntc + cq * QWC + c0, a);
+      }
+      xz2[cq * kRows + r] = zloc;
+    }
+    cp_async_wait_all();
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    if (e0 == 0) PHASE_MARK(15);
+#pragma unroll
+    for (int u = 0; u < NQ; ++u) z_run += xz2[u * kRows + r];
+
+    // ---- O += A_c . Vbar_c; then stage the next chunk's codes (the logits MMA of this chunk is done)
+    const int e_next = e0 + CHW;
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t aa = smem_u32(CA), va = smem_u32(Vs);
+      for (int k = 0; k < np16 / 16; ++k)
+        umma_bf16(tmem_base + CT, umma_desc_sw128(aa + (k / 4) * kRows * 128 + (k % 4) * 32),
+                  umma_desc_sw128(va + (k / 4) * D * 128 + (k % 4) * 32), idesc_o, true);
+      umma_commit(bar_pv);
+    }
+    if (e_next < PC) {
+      ncols = min(PC - e_next, CHW);
+      np16 = (ncols + 15) & ~15;
+      gather_codes(e_next);
+      cp_async_wait_all();
+      fence_proxy_async();
+      tc_fence_before();
+      __syncthreads();
+      if (tid == 0) {
+        tc_fence_after();
+        const uint32_t idesc = umma_idesc_bf16(kRows, np16);
+        const uint32_t qa = smem_u32(Qs), ca = smem_u32(CC);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)
+          umma_bf16(tmem_base, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
+                    umma_desc_sw128(ca + (k / 4) * np16 * 128 + (k % 4) * 32), idesc, k > 0);
+        umma_commit(bar_s);
+      }
+    }
   }
 
   // ---- epilogue: Y = O / z
+  PHASE_MARK(26);
   const bool o_ok = mbar_wait(bar_pv, ph_pv, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
   tc_fence_after();
+  PHASE_MARK(27);
   if (o_ok) {
     // tcgen05.ld is warp-collective: every lane loads, only rows inside the tensor store.
     const float inv = 1.f / z_run;
-    __nv_bfloat16* yrow = p.Y + ((size_t)bh * p.Nq + i0 + r) * D + hf * (D / 2);
-    for (int c0 = 0; c0 < D / 2; c0 += 16) {
+    __nv_bfloat16* yrow = p.Y + ((size_t)bh * p.Nq + i0 + r) * D + cq * (D / NQ);
+    for (int c0 = 0; c0 < D / NQ; c0 += 16) {
       float o[16];
       tmem_ld16(t_o + c0, o);
       uint32_t pk[8];
@@ -424,18 +603,31 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
     }
   }
+  PHASE_MARK(28);
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+  PHASE_MARK(29);
 }
 
-size_t attend_smem(int D, int CT) {
-  const int subA = (CT + 63) / 64;
+size_t attend_smem(int D, int CT, int CHW) {
+  const int subA = CT / 64;
   const size_t ca = (size_t)max(CT * D * 2, subA * kRows * 128);
-  size_t b = 1024 + (size_t)(D / 64) * kRows * 128 + ca + (size_t)subA * D * 128;
-  b += sizeof(float) * ((size_t)CT + 256 + 4 * (size_t)CT + 6 * kRows);
-  b += sizeof(int) * 256 + sizeof(uint32_t) * 8 + sizeof(uint64_t) * 4 + 2 * sizeof(uint32_t) + 256;
+  size_t b = 1024 + (size_t)(D / 64) * kRows * 128 + ca + (size_t)subA * D * 128 + (size_t)CHW * D * 2;
+  b += sizeof(float) * (3 * (size_t)CT + 2 * (size_t)CHW + 256 + 4 * (size_t)CT + 12 * kRows);
+  b += sizeof(int) * 256 + sizeof(uint32_t) * 18 + sizeof(uint64_t) * 4 + 2 * sizeof(uint32_t);
   return b + 64;
+}
+
+template <int D, int NQ, int CT>
+avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUtensorMap& tmVpT,
+                     const AttendParams& a, unsigned BH, size_t smem, cudaStream_t st) {
+  auto kern = tc_attend_kernel<D, NQ, CT>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return AVQ_ERR_CUDA;
+  dim3 grid(a.nblk, BH);
+  kern<<<grid, 128 * NQ, smem, st>>>(tmQ, tmCp, tmVpT, a);
+  return cuda_ok(cudaGetLastError());
 }
 
 template <int D>
@@ -473,23 +665,34 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
   a.status_word = status_word;
   a.H = p.H; a.Nq = p.Nq; a.M = p.M; a.C = p.C; a.P = P;
   a.nblk = (p.Nq + kRows - 1) / kRows;
-  int CT = 32;
-  while (CT < p.M) CT <<= 1;
-  a.CT = CT;
+  const int CT = p.M <= 64 ? 64 : (p.M <= 128 ? 128 : 256);
+  const int CHW = CT < 128 ? CT : 128;
+  a.logC = p.C == 8 ? 3 : 2;
   uint32_t cols = 32;
   while ((int)cols < CT + D) cols <<= 1;
   a.tmem_cols = cols;
   a.scale_log2e = p.scale * 1.4426950408889634f;
-  const size_t smem = attend_smem(D, CT);
-  auto kern = tc_attend_kernel<D>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return AVQ_ERR_CUDA;
-  dim3 grid(a.nblk, (unsigned)BH);
-  kern<<<grid, kThreads, smem, st>>>(tmQ, tmCp, tmVpT, a);
-  return cuda_ok(cudaGetLastError());
+  const size_t smem = attend_smem(D, CT, CHW);
+  // Threads per query row follow from how many CTAs can share an SM (TMEM columns, shared memory):
+  // four small CTAs of 128 threads, two of 256, or one of 512.
+  const unsigned bh = (unsigned)BH;
+  if (D == 64) {
+    if (CT == 64) return launch_nq<D, 1, 64>(tmQ, tmCp, tmVpT, a, bh, smem, st);
+    if (CT == 128) return launch_nq<D, 2, 128>(tmQ, tmCp, tmVpT, a, bh, smem, st);
+    return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, a, bh, smem, st);
+  }
+  if (CT == 64) return launch_nq<D, 2, 64>(tmQ, tmCp, tmVpT, a, bh, smem, st);
+  if (CT == 128) return launch_nq<D, 4, 128>(tmQ, tmCp, tmVpT, a, bh, smem, st);
+  return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, a, bh, smem, st);
 }
 
 }  // namespace
+
+#ifdef AVQ_PHASE_DEBUG
+extern "C" __attribute__((visibility("default"))) int avq_debug_phase_clocks(long long* host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, g_phase_clocks, sizeof(long long) * 64 * 32);
+}
+#endif
 
 avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc, const float* np_,
                      const float* nc, const void* VpT, const void* VcT, int32_t P, void* Y, int32_t* topp_out,
