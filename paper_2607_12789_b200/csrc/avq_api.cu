@@ -58,12 +58,13 @@ Layout make_layout(const avq_problem& p, int32_t /*P*/, int32_t /*block_q*/) {
   size_t off = 256;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   L.header = 0;
+  L.Vc = take(sizeof(float) * BH * p.M * p.C * p.d);
+  L.nc = take(sizeof(float) * BH * p.M * p.C);
+  L.zero_end = off;
   L.parent_idx = take(sizeof(int32_t) * BH * p.Nk);
   L.child_idx = take(sizeof(int32_t) * BH * p.Nk);
   L.Vp = take(sizeof(float) * BH * p.M * p.d);
   L.np = take(sizeof(float) * BH * p.M);
-  L.Vc = take(sizeof(float) * BH * p.M * p.C * p.d);
-  L.nc = take(sizeof(float) * BH * p.M * p.C);
   if (use_tensor_path(p)) {
     L.VpT = take(2 * BH * p.M * p.d);
     L.VcT = take(2 * BH * p.M * p.C * p.d);
@@ -121,7 +122,7 @@ avq_status avq_aggregate(const avq_problem* prob, const void* V, const int32_t* 
     return AVQ_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (use_tensor_path(*prob))
-    return tc_aggregate(*prob, V, parent_idx, child_idx, Vp, np_, Vc, nc, nullptr, nullptr, st);
+    return tc_aggregate(*prob, V, parent_idx, child_idx, Vp, np_, Vc, nc, nullptr, nullptr, false, st);
   return simt_aggregate(*prob, V, parent_idx, child_idx, Vp, np_, Vc, nc, st);
 }
 
@@ -178,12 +179,14 @@ avq_status avq_forward(const avq_problem* prob, const void* Q, const void* K, co
   const avq_problem& p = *prob;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Regions r = carve(workspace, L);
-  if (cudaMemsetAsync(r.status_word, 0, 256, st) != cudaSuccess) return AVQ_ERR_CUDA;
   if (use_tensor_path(p)) {
+    // one memset: status header, leaf sums and leaf counts are adjacent
+    if (cudaMemsetAsync(workspace, 0, L.zero_end, st) != cudaSuccess) return AVQ_ERR_CUDA;
     s = tc_assign(p, K, Cp, Cc, r.pidx, r.cidx, r.status_word, st);
     if (s != AVQ_OK) return s;
-    s = tc_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, r.VpT, r.VcT, st);
+    s = tc_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, r.VpT, r.VcT, true, st);
   } else {
+    if (cudaMemsetAsync(r.status_word, 0, 256, st) != cudaSuccess) return AVQ_ERR_CUDA;
     s = simt_assign(p, K, Cp, Cc, r.pidx, r.cidx, st);
     if (s != AVQ_OK) return s;
     s = simt_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, st);

@@ -12,12 +12,13 @@ namespace avq {
 // Byte offsets of the regions of an avq_forward workspace.
 struct Layout {
   size_t header = 0;       // 256 bytes; int32 status word at offset 0
+  size_t Vc = 0;           // f32 [B,H,M,C,d]   header, Vc and nc are adjacent: one memset clears them
+  size_t nc = 0;           // f32 [B,H,M,C]
+  size_t zero_end = 0;     // end of the region that must be zero before aggregation
   size_t parent_idx = 0;   // int32 [B,H,Nk]
   size_t child_idx = 0;    // int32 [B,H,Nk]
   size_t Vp = 0;           // f32 [B,H,M,d]
   size_t np = 0;           // f32 [B,H,M]
-  size_t Vc = 0;           // f32 [B,H,M,C,d]
-  size_t nc = 0;           // f32 [B,H,M,C]
   size_t VpT = 0;          // bf16 [B,H,d,M]      (tensor-core path only)
   size_t VcT = 0;          // bf16 [B,H,M,d,C]    (tensor-core path only)
   size_t total = 0;
@@ -51,7 +52,7 @@ avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const 
                      int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, cudaStream_t st);
 avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
                         const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc,
-                        void* VpT, void* VcT, cudaStream_t st);
+                        void* VpT, void* VcT, bool pre_zeroed, cudaStream_t st);
 avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc,
                      const float* np_, const float* nc, const void* VpT, const void* VcT, int32_t P,
                      void* Y, int32_t* topp_out, float* importance_out, int32_t* status_word,

@@ -1,6 +1,6 @@
 // Value aggregation for the bf16 path (Eq. "aggregates"; the scatter steps of Algorithm 1).
 //
-// leaf_scatter_kernel  one warp per key: the key's V row is added to the sum of its leaf
+// leaf_scatter_kernel  one warp per 8 keys: each key's V row is added to the sum of its leaf
 //                      codeword (parent, child) with vector reductions to global memory, and
 //                      the leaf's count is bumped.  Only the leaf level is scattered.
 // finalize_kernel      per parent: Vp = sum over its children (every key sits in exactly one
@@ -8,14 +8,19 @@
 //                      the bf16 operand copies the attention kernel stages with TMA:
 //                        VpT [B,H,d,M]    value sums with the codeword index fastest
 //                        VcT [B,H,M,d,C]  per parent a contiguous d x C block, child fastest
+#include <type_traits>
+
 #include "avq_tc_common.cuh"
 
 namespace avq {
 namespace {
 
 constexpr int kScatterThreads = 256;
-constexpr int kKeysPerCta = 256;
+constexpr int kKeysPerWarp = 8;
+constexpr int kKeysPerCta = kKeysPerWarp * (kScatterThreads / 32);
 
+// One warp = 8 consecutive keys: their indices are read with one coalesced load and broadcast by
+// shuffle, the 8 value rows are loaded before the first reduction is issued.
 template <int D>
 __global__ void __launch_bounds__(kScatterThreads)
 leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restrict__ pidx,
@@ -23,78 +28,100 @@ leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restri
                     int Nk, int M, int C) {
   const int bh = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int j0 = blockIdx.x * kKeysPerCta;
-  const int j1 = min(Nk, j0 + kKeysPerCta);
+  const int j0 = blockIdx.x * kKeysPerCta + warp * kKeysPerWarp;
+  if (j0 >= Nk) return;
   const size_t kb = (size_t)bh * Nk;
-  for (int j = j0 + warp; j < j1; j += kScatterThreads / 32) {
-    const int a = __ldg(pidx + kb + j);
-    const int c = __ldg(cidx + kb + j);
-    const size_t leaf = ((size_t)bh * M + a) * C + c;
-    float* dst = Vc + leaf * D;
-    const __nv_bfloat16* v = V + (kb + j) * D;
-    if constexpr (D == 128) {
-      const uint2 u = __ldg(reinterpret_cast<const uint2*>(v) + lane);
-      float4 f = make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u),
-                             __uint_as_float(u.y << 16), __uint_as_float(u.y & 0xFFFF0000u));
-      atomicAdd(reinterpret_cast<float4*>(dst) + lane, f);
-    } else {
-      const uint32_t u = __ldg(reinterpret_cast<const uint32_t*>(v) + lane);
-      float2 f = make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
-      atomicAdd(reinterpret_cast<float2*>(dst) + lane, f);
-    }
-    if (lane == 0) atomicAdd(nc + leaf, 1.0f);
+  int leaf_l = -1;
+  if (lane < kKeysPerWarp && j0 + lane < Nk) {
+    const int a = __ldg(pidx + kb + j0 + lane);
+    const int c = __ldg(cidx + kb + j0 + lane);
+    leaf_l = a * C + c;
   }
+  using Vec = typename std::conditional<D == 128, uint2, uint32_t>::type;
+  Vec v[kKeysPerWarp];
+#pragma unroll
+  for (int t = 0; t < kKeysPerWarp; ++t)
+    if (j0 + t < Nk) v[t] = __ldg(reinterpret_cast<const Vec*>(V + (kb + j0 + t) * D) + lane);
+#pragma unroll
+  for (int t = 0; t < kKeysPerWarp; ++t) {
+    const int leaf = __shfl_sync(0xffffffffu, leaf_l, t);
+    if (leaf < 0) continue;                           // past the end (warp-uniform)
+    float* dst = Vc + ((size_t)bh * M * C + leaf) * D;
+    if constexpr (D == 128) {
+      const uint2 u = v[t];
+      atomicAdd(reinterpret_cast<float4*>(dst) + lane,
+                make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u),
+                            __uint_as_float(u.y << 16), __uint_as_float(u.y & 0xFFFF0000u)));
+    } else {
+      const uint32_t u = v[t];
+      atomicAdd(reinterpret_cast<float2*>(dst) + lane,
+                make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u)));
+    }
+  }
+  if (leaf_l >= 0) atomicAdd(nc + (size_t)bh * M * C + leaf_l, 1.0f);
 }
 
 // One CTA: 8 consecutive parents of one (batch, head); thread k owns head-dimension index k.
-template <int D>
+// All loads of four parents are issued before their first use.
+template <int D, int C>
 __global__ void __launch_bounds__(D)
 finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, float* __restrict__ Vp,
                 float* __restrict__ np_, __nv_bfloat16* __restrict__ VpT, __nv_bfloat16* __restrict__ VcT,
-                int M, int C) {
+                int M) {
   const int bh = blockIdx.y, m0 = blockIdx.x * 8, k = threadIdx.x;
   __align__(16) __nv_bfloat16 pk[8];
 #pragma unroll
-  for (int mm = 0; mm < 8; ++mm) {
-    const int m = m0 + mm;
-    const float* src = Vc + (((size_t)bh * M + m) * C) * D + k;
-    __align__(16) __nv_bfloat16 ck[8];
-    float s = 0.f;
-    for (int c = 0; c < C; ++c) {
-      const float x = src[(size_t)c * D];
-      s += x;
-      ck[c] = __float2bfloat16_rn(x);
-    }
-    Vp[((size_t)bh * M + m) * D + k] = s;
-    pk[mm] = __float2bfloat16_rn(s);
-    if (VcT) {
-      __nv_bfloat16* dst = VcT + (((size_t)bh * M + m) * D + k) * C;
-      if (C == 8) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(ck);
-      else *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(ck);
+  for (int g = 0; g < 2; ++g) {
+    float x[4][C];
+#pragma unroll
+    for (int mm = 0; mm < 4; ++mm)
+#pragma unroll
+      for (int c = 0; c < C; ++c)
+        x[mm][c] = Vc[((((size_t)bh * M + m0 + g * 4 + mm) * C) + c) * D + k];
+#pragma unroll
+    for (int mm = 0; mm < 4; ++mm) {
+      const int m = m0 + g * 4 + mm;
+      __align__(16) __nv_bfloat16 ck[C];
+      float s = 0.f;
+#pragma unroll
+      for (int c = 0; c < C; ++c) {
+        s += x[mm][c];
+        ck[c] = __float2bfloat16_rn(x[mm][c]);
+      }
+      Vp[((size_t)bh * M + m) * D + k] = s;
+      pk[g * 4 + mm] = __float2bfloat16_rn(s);
+      if (VcT) {
+        __nv_bfloat16* dst = VcT + (((size_t)bh * M + m) * D + k) * C;
+        if (C == 8) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(ck);
+        else *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(ck);
+      }
     }
   }
   if (VpT) *reinterpret_cast<uint4*>(VpT + ((size_t)bh * D + k) * M + m0) = *reinterpret_cast<const uint4*>(pk);
   if (k < 8) {
     const int m = m0 + k;
     float s = 0.f;
+#pragma unroll
     for (int c = 0; c < C; ++c) s += nc[((size_t)bh * M + m) * C + c];
     np_[(size_t)bh * M + m] = s;
   }
 }
 
-template <int D>
+template <int D, int C>
 avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const int32_t* cidx, float* Vp,
-               float* np_, float* Vc, float* nc, void* VpT, void* VcT, cudaStream_t st) {
+               float* np_, float* Vc, float* nc, void* VpT, void* VcT, bool pre_zeroed, cudaStream_t st) {
   const unsigned BH = (unsigned)(p.B * p.H);
-  if (cudaMemsetAsync(Vc, 0, sizeof(float) * (size_t)BH * p.M * p.C * D, st) != cudaSuccess) return AVQ_ERR_CUDA;
-  if (cudaMemsetAsync(nc, 0, sizeof(float) * (size_t)BH * p.M * p.C, st) != cudaSuccess) return AVQ_ERR_CUDA;
+  if (!pre_zeroed) {
+    if (cudaMemsetAsync(Vc, 0, sizeof(float) * (size_t)BH * p.M * C * D, st) != cudaSuccess) return AVQ_ERR_CUDA;
+    if (cudaMemsetAsync(nc, 0, sizeof(float) * (size_t)BH * p.M * C, st) != cudaSuccess) return AVQ_ERR_CUDA;
+  }
   dim3 g1((p.Nk + kKeysPerCta - 1) / kKeysPerCta, BH);
   leaf_scatter_kernel<D><<<g1, kScatterThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(V), pidx, cidx, Vc,
-                                                         nc, p.Nk, p.M, p.C);
+                                                         nc, p.Nk, p.M, C);
   if (cudaGetLastError() != cudaSuccess) return AVQ_ERR_CUDA;
   dim3 g2(p.M / 8, BH);
-  finalize_kernel<D><<<g2, D, 0, st>>>(Vc, nc, Vp, np_, static_cast<__nv_bfloat16*>(VpT),
-                                       static_cast<__nv_bfloat16*>(VcT), p.M, p.C);
+  finalize_kernel<D, C><<<g2, D, 0, st>>>(Vc, nc, Vp, np_, static_cast<__nv_bfloat16*>(VpT),
+                                          static_cast<__nv_bfloat16*>(VcT), p.M);
   return cuda_ok(cudaGetLastError());
 }
 
@@ -102,9 +129,12 @@ avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const i
 
 avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
                         const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc, void* VpT,
-                        void* VcT, cudaStream_t st) {
-  return p.d == 64 ? run<64>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, VpT, VcT, st)
-                   : run<128>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, VpT, VcT, st);
+                        void* VcT, bool pre_zeroed, cudaStream_t st) {
+  if (p.d == 64)
+    return p.C == 4 ? run<64, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, VpT, VcT, pre_zeroed, st)
+                    : run<64, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, VpT, VcT, pre_zeroed, st);
+  return p.C == 4 ? run<128, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, VpT, VcT, pre_zeroed, st)
+                  : run<128, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, VpT, VcT, pre_zeroed, st);
 }
 
 }  // namespace avq

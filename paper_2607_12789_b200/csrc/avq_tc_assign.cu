@@ -1,13 +1,15 @@
 // Tensor-core key assignment (Algorithm 1, parent and child argmin) for bf16 inputs.
 //
-// One CTA takes 128 consecutive keys of one (batch, head).  TMA stages the key tile and the
-// head's parent codebook in shared memory (K-major, 128-byte swizzle); one elected thread
-// issues the tcgen05 MMA chain  D[128 x M] = K_tile . Cp^T  into TMEM.  Each of the 128
-// threads then owns one key (one TMEM lane): it reads its row of dot products, forms
-// ||c||^2 - 2 k.c, keeps the best and the runner-up, and - only when those two are closer
-// than the MMA's rounding can separate - re-evaluates all M distances in float64 in the direct
-// form.  The child argmin over the C children of the winner runs on CUDA cores (2 C d
-// flops per key; a second MMA over all M C children would cost C times the parent GEMM).
+// One CTA takes 128 consecutive keys of one (batch, head), 8 warps.  TMA stages the key tile and the
+// head's parent codebook in shared memory (K-major, 128-byte swizzle); one elected thread issues the
+// tcgen05 MMA chain  D[128 x M] = K_tile . Cp^T  into TMEM.
+//   parent   two threads per key (column halves) read their TMEM lane, form ||c||^2 - 2 k.c and keep
+//            the best and the runner-up; the halves are merged in shared memory.  Only when best and
+//            runner-up are closer than the MMA's rounding can separate are all M distances redone in
+//            float64 in the direct form (lowest index wins ties).
+//   child    the two threads of a key split the C children of its parent and evaluate the direct form
+//            sum (k - c)^2 in fp32 on CUDA cores (2 C d flops per key; a second MMA over all M C
+//            children would cost C times the parent GEMM).  Same float64 recheck for near-ties.
 #include "avq_tc_common.cuh"
 
 namespace avq {
@@ -16,44 +18,52 @@ namespace {
 using namespace tc;
 
 constexpr int kKeys = 128;
+constexpr int kThreadsA = 256;
+
+#ifdef AVQ_PHASE_DEBUG
+__device__ long long g_assign_clocks[64 * 16];
+#define APHASE(i) do { if (threadIdx.x == 0 && blockIdx.x < 8 && blockIdx.y < 8) \
+    g_assign_clocks[(blockIdx.y * 8 + blockIdx.x) * 16 + (i)] = clock64(); } while (0)
+#else
+#define APHASE(i) do { } while (0)
+#endif
 
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
 
-template <int D>
-__device__ double exact_dist_regs(const uint32_t (&kreg)[D / 2], const __nv_bfloat16* c) {
-  double s = 0.0;
-#pragma unroll 4
-  for (int q = 0; q < D / 2; ++q) {
-    const double a = (double)bf_lo(kreg[q]) - (double)__bfloat162float(c[2 * q]);
-    const double b = (double)bf_hi(kreg[q]) - (double)__bfloat162float(c[2 * q + 1]);
-    s += a * a;
-    s += b * b;
-  }
-  return s;
-}
-
-template <int D>
-__device__ float direct_dist_regs(const uint32_t (&kreg)[D / 2], const __nv_bfloat16* c) {
-  const uint4* c4 = reinterpret_cast<const uint4*>(c);
+// sum over 8 bf16 pairs of (a - b)^2 for two packed 16-byte chunks
+__device__ __forceinline__ float sqdiff8(const uint4& a, const uint4& b) {
+  const uint32_t x[4] = {a.x, a.y, a.z, a.w}, y[4] = {b.x, b.y, b.z, b.w};
   float s = 0.f;
 #pragma unroll
-  for (int q = 0; q < D / 8; ++q) {
-    const uint4 v = __ldg(c4 + q);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float a = bf_lo(kreg[4 * q + e]) - bf_lo(w[e]);
-      const float b = bf_hi(kreg[4 * q + e]) - bf_hi(w[e]);
-      s = fmaf(a, a, s);
-      s = fmaf(b, b, s);
-    }
+  for (int e = 0; e < 4; ++e) {
+    const float d0 = bf_lo(x[e]) - bf_lo(y[e]);
+    const float d1 = bf_hi(x[e]) - bf_hi(y[e]);
+    s = fmaf(d0, d0, s);
+    s = fmaf(d1, d1, s);
+  }
+  return s;
+}
+
+// element `col` (0..D-1) of key row `row` in the swizzled key tile
+template <int D>
+__device__ __forceinline__ float key_elem(const unsigned char* Ks, int row, int col) {
+  const unsigned char* sub = Ks + (col >> 6) * (kKeys * 128);
+  return __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sub + sw128_offset(row, col & 63)));
+}
+
+template <int D>
+__device__ double exact_dist_smem(const unsigned char* Ks, int row, const __nv_bfloat16* c) {
+  double s = 0.0;
+  for (int k = 0; k < D; ++k) {
+    const double t = (double)key_elem<D>(Ks, row, k) - (double)__bfloat162float(c[k]);
+    s += t * t;
   }
   return s;
 }
 
 template <int D>
-__global__ void __launch_bounds__(kKeys)
+__global__ void __launch_bounds__(kThreadsA, 2)
 tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmCp,
                  const __nv_bfloat16* __restrict__ Cp, const __nv_bfloat16* __restrict__ Cc,
                  int32_t* __restrict__ pidx, int32_t* __restrict__ cidx, int H, int Nk, int M, int C,
@@ -65,21 +75,36 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   unsigned char* Ks = smem;                          // kSub x [128 x 128 B]
   unsigned char* Cs = Ks + kSub * kKeys * 128;       // kSub x [M x 128 B]
   float* cnorm = reinterpret_cast<float*>(Cs + kSub * M * 128);   // [M]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(cnorm + M);        // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* xd1 = cnorm + M;                            // [2][128] best distance of each column half
+  float* xd2 = xd1 + 2 * kKeys;                      // [2][128] runner-up
+  float* xkn = xd2 + 2 * kKeys;                      // [2][128] halves of ||k||^2
+  int* xi1 = reinterpret_cast<int*>(xkn + 2 * kKeys);   // [2][128] index of the best
+  int* par = xi1 + 2 * kKeys;                        // [128] final parent of each key
+  int* chi = par + kKeys;                            // [128] final child of each key
+  uint32_t* cmax_bits = reinterpret_cast<uint32_t*>(chi + kKeys);   // max ||c||^2 (non-negative float bits)
+  uint32_t* tmem_slot = cmax_bits + 1;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tmem_slot + 1);      // [2]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2);
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int q = warp & 3, hf = warp >> 2, r = q * 32 + lane;
   const int bh = blockIdx.y, h = bh % H;
-  const int j0 = blockIdx.x * kKeys, j = j0 + tid;
+  const int j0 = blockIdx.x * kKeys;
+  const int MH = M >> 1;                             // columns per half (multiple of 16: M % 32 == 0)
 
+  APHASE(0);
   if (tid == 0) {
     mbar_init(&bars[0], 1);
     mbar_init(&bars[1], 1);
     mbar_fence_init();
     *abort_flag = 0;
-    prefetch_tmap(&tmK);
-    prefetch_tmap(&tmCp);
+    *cmax_bits = 0;
+    mbar_expect_tx(&bars[0], (uint32_t)(kSub * (kKeys + M) * 128));
+#pragma unroll
+    for (int s = 0; s < kSub; ++s) {
+      tma_load_3d(Ks + s * kKeys * 128, &tmK, s * 64, j0, bh, &bars[0]);
+      tma_load_2d(Cs + s * M * 128, &tmCp, s * 64, h * M, &bars[0]);
+    }
   }
   if (warp == 0) {
     tmem_alloc(tmem_slot, tmem_cols);
@@ -89,124 +114,174 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  APHASE(1);
 
-  if (tid == 0) {
-    mbar_expect_tx(&bars[0], (uint32_t)(kSub * (kKeys + M) * 128));
-#pragma unroll
-    for (int s = 0; s < kSub; ++s) {
-      tma_load_3d(Ks + s * kKeys * 128, &tmK, s * 64, j0, bh, &bars[0]);
-      tma_load_2d(Cs + s * M * 128, &tmCp, s * 64, h * M, &bars[0]);
-    }
-  }
   const bool loaded = mbar_wait(&bars[0], 0, abort_flag, status_word, DEV_TIMEOUT_ASSIGN);
-
+  APHASE(2);
   if (tid == 0 && loaded) {
     tc_fence_after();
     const uint32_t idesc = umma_idesc_bf16(kKeys, M);
     const uint32_t ka = smem_u32(Ks), ca = smem_u32(Cs);
 #pragma unroll
-    for (int k = 0; k < D / 16; ++k) {
-      const uint64_t ad = umma_desc_sw128(ka + (k / 4) * kKeys * 128 + (k % 4) * 32);
-      const uint64_t bd = umma_desc_sw128(ca + (k / 4) * M * 128 + (k % 4) * 32);
-      umma_bf16(tmem_base, ad, bd, idesc, k > 0);
-    }
+    for (int k = 0; k < D / 16; ++k)
+      umma_bf16(tmem_base, umma_desc_sw128(ka + (k / 4) * kKeys * 128 + (k % 4) * 32),
+                umma_desc_sw128(ca + (k / 4) * M * 128 + (k % 4) * 32), idesc, k > 0);
     umma_commit(&bars[1]);
   }
 
-  // ||c_m||^2 from the staged codebook, and this thread's key row into registers
-  for (int m = tid; m < M; m += kKeys) {
+  // ||c_m||^2 from the staged codebook (and its maximum), half of ||k||^2 per thread
+  for (int m = tid; m < M; m += kThreadsA) {
     float s = 0.f;
 #pragma unroll
     for (int sub = 0; sub < kSub; ++sub) {
-      const unsigned char* row = Cs + sub * M * 128;
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {
-        const uint4 v = *reinterpret_cast<const uint4*>(row + sw128_offset(m, ch * 8));
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        const uint4 v = *reinterpret_cast<const uint4*>(Cs + sub * M * 128 + sw128_offset(m, ch * 8));
+        const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          s = fmaf(bf_lo(w[e]), bf_lo(w[e]), s);
-          s = fmaf(bf_hi(w[e]), bf_hi(w[e]), s);
+          s = fmaf(bf_lo(wv[e]), bf_lo(wv[e]), s);
+          s = fmaf(bf_hi(wv[e]), bf_hi(wv[e]), s);
         }
       }
     }
     cnorm[m] = s;
+    atomicMax(cmax_bits, __float_as_uint(s));
   }
-  uint32_t kreg[D / 2];
-  float knorm = 0.f;
+  {
+    float s = 0.f;
+    constexpr int kChunksHalf = D / 16;              // 16-byte chunks in half a row
 #pragma unroll
-  for (int sub = 0; sub < kSub; ++sub) {
-#pragma unroll
-    for (int ch = 0; ch < 8; ++ch) {
-      const uint4 v = *reinterpret_cast<const uint4*>(Ks + sub * kKeys * 128 + sw128_offset(tid, ch * 8));
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    for (int cc = 0; cc < kChunksHalf; ++cc) {
+      const int ch = hf * kChunksHalf + cc;          // chunk index in the row, 0 .. D/8-1
+      const uint4 v = *reinterpret_cast<const uint4*>(Ks + (ch >> 3) * kKeys * 128 + sw128_offset(r, (ch & 7) * 8));
+      const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        kreg[sub * 32 + ch * 4 + e] = w[e];
-        knorm = fmaf(bf_lo(w[e]), bf_lo(w[e]), knorm);
-        knorm = fmaf(bf_hi(w[e]), bf_hi(w[e]), knorm);
+        s = fmaf(bf_lo(wv[e]), bf_lo(wv[e]), s);
+        s = fmaf(bf_hi(wv[e]), bf_hi(wv[e]), s);
       }
     }
+    xkn[hf * kKeys + r] = s;
   }
-  __syncthreads();   // cnorm visible
+  APHASE(3);
+  __syncthreads();   // cnorm, cmax visible
+  APHASE(4);
 
   const bool done = mbar_wait(&bars[1], 0, abort_flag, status_word, DEV_TIMEOUT_ASSIGN);
   tc_fence_after();
+  APHASE(5);
 
-  float d1 = INFINITY, d2 = INFINITY, cmax = 0.f;
-  int i1 = 0;
-  if (done) {
-    const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
-    for (int c0 = 0; c0 < M; c0 += 16) {
+  // ---- parent argmin over this thread's half of the columns
+  {
+    float d1 = INFINITY, d2 = INFINITY;
+    int i1 = 0;
+    const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(hf * MH);
+    for (int c0 = 0; c0 < MH; c0 += 16) {
       float dot[16];
-      tmem_ld16(trow + c0, dot);
+      tmem_ld16(trow + c0, dot);                     // warp-collective: executed by every lane
+      const float4* cn4 = reinterpret_cast<const float4*>(cnorm + hf * MH + c0);
 #pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        const float cn = cnorm[c0 + e];
-        const float dist = fmaf(-2.f, dot[e], cn);
-        cmax = fmaxf(cmax, cn);
-        if (dist < d1) { d2 = d1; d1 = dist; i1 = c0 + e; }
-        else if (dist < d2) { d2 = dist; }
+      for (int u = 0; u < 4; ++u) {
+        const float4 cn = cn4[u];
+        const float dist[4] = {fmaf(-2.f, dot[4 * u], cn.x), fmaf(-2.f, dot[4 * u + 1], cn.y),
+                               fmaf(-2.f, dot[4 * u + 2], cn.z), fmaf(-2.f, dot[4 * u + 3], cn.w)};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          d2 = fminf(d2, fmaxf(dist[e], d1));        // runner-up: second smallest so far
+          if (dist[e] < d1) { d1 = dist[e]; i1 = hf * MH + c0 + 4 * u + e; }
+        }
       }
     }
+    xd1[hf * kKeys + r] = d1;
+    xd2[hf * kKeys + r] = d2;
+    xi1[hf * kKeys + r] = i1;
   }
+  APHASE(6);
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, tmem_cols);
-  if (j >= Nk || !done) return;
+  APHASE(7);
 
+  // ---- merge the halves (the lower half holds the lower indices, so it wins ties); recheck near-ties
   const __nv_bfloat16* Cph = Cp + (size_t)h * M * D;
-  // The MMA accumulates k.c in fp32: its error is a small multiple of 2^-24 * ||k|| * ||c||, which
-  // 2e-4 * (||k||^2 + max ||c||^2) bounds with a wide margin.
-  if (M > 1 && !(d2 - d1 > 2e-4f * (knorm + cmax))) {
-    double best = INFINITY;
-    int bi = 0;
-    for (int m = 0; m < M; ++m) {
-      const double s = exact_dist_regs<D>(kreg, Cph + (size_t)m * D);
-      if (s < best) { best = s; bi = m; }
+  if (hf == 0) {
+    const float a1 = xd1[r], a2 = xd2[r], b1 = xd1[kKeys + r], b2 = xd2[kKeys + r];
+    int i1 = (b1 < a1) ? xi1[kKeys + r] : xi1[r];
+    const float d1 = fminf(a1, b1);
+    const float d2 = fminf(fmaxf(a1, b1), fminf(a2, b2));
+    const float knorm = xkn[r] + xkn[kKeys + r];
+    const float cmax = __uint_as_float(*cmax_bits);
+    // The MMA accumulates k.c in fp32: its error is a small multiple of 2^-24 * ||k|| * ||c||, which
+    // 2e-4 * (||k||^2 + max ||c||^2) bounds with a wide margin.
+    if (done && j0 + r < Nk && !(d2 - d1 > 2e-4f * (knorm + cmax))) {
+      double best = INFINITY;
+      int bi = 0;
+      for (int m = 0; m < M; ++m) {
+        const double s = exact_dist_smem<D>(Ks, r, Cph + (size_t)m * D);
+        if (s < best) { best = s; bi = m; }
+      }
+      i1 = bi;
     }
-    i1 = bi;
+    par[r] = i1;
   }
+  __syncthreads();
+  APHASE(8);
 
-  const __nv_bfloat16* Cch = Cc + ((size_t)h * M + i1) * C * D;
-  float e1 = INFINITY, e2 = INFINITY;
-  int c1 = 0;
-  for (int c = 0; c < C; ++c) {
-    const float s = direct_dist_regs<D>(kreg, Cch + (size_t)c * D);
-    if (s < e1) { e2 = e1; e1 = s; c1 = c; }
-    else if (s < e2) { e2 = s; }
-  }
-  if (C > 1 && !(e2 - e1 > 1e-4f * e2)) {
-    double best = INFINITY;
-    int bi = 0;
-    for (int c = 0; c < C; ++c) {
-      const double s = exact_dist_regs<D>(kreg, Cch + (size_t)c * D);
-      if (s < best) { best = s; bi = c; }
+  // ---- child argmin: the two threads of a key take half of the C children each (fp32 direct form),
+  // eight 16-byte loads in flight per thread; the halves are merged like the parents'
+  {
+    const int a = par[r];
+    const int CH = C >> 1;                           // children per thread (C is 4 or 8)
+    const __nv_bfloat16* Cch = Cc + (((size_t)h * M + a) * C + (size_t)hf * CH) * D;
+    float e1 = INFINITY, e2 = INFINITY;
+    int c1 = 0;
+    for (int c = 0; c < CH; ++c) {
+      const uint4* src = reinterpret_cast<const uint4*>(Cch + (size_t)c * D);
+      float s = 0.f;
+#pragma unroll
+      for (int g = 0; g < D / 64; ++g) {             // 8 chunks (64 elements) at a time
+        uint4 cv[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) cv[t] = __ldg(src + g * 8 + t);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          const uint4 kv = *reinterpret_cast<const uint4*>(Ks + g * kKeys * 128 + sw128_offset(r, t * 8));
+          s += sqdiff8(kv, cv[t]);
+        }
+      }
+      e2 = fminf(e2, fmaxf(s, e1));
+      if (s < e1) { e1 = s; c1 = hf * CH + c; }
     }
-    c1 = bi;
+    xd1[hf * kKeys + r] = e1;
+    xd2[hf * kKeys + r] = e2;
+    xi1[hf * kKeys + r] = c1;
   }
-  pidx[(size_t)bh * Nk + j] = i1;
-  cidx[(size_t)bh * Nk + j] = c1;
+  __syncthreads();
+  if (hf == 0) {
+    const float a1 = xd1[r], a2 = xd2[r], b1 = xd1[kKeys + r], b2 = xd2[kKeys + r];
+    int c1 = (b1 < a1) ? xi1[kKeys + r] : xi1[r];
+    const float e1 = fminf(a1, b1);
+    const float e2 = fminf(fmaxf(a1, b1), fminf(a2, b2));
+    if (done && j0 + r < Nk && !(e2 - e1 > 1e-4f * e2)) {
+      const __nv_bfloat16* Cch = Cc + ((size_t)h * M + par[r]) * C * D;
+      double best = INFINITY;
+      int bi = 0;
+      for (int c = 0; c < C; ++c) {
+        const double s = exact_dist_smem<D>(Ks, r, Cch + (size_t)c * D);
+        if (s < best) { best = s; bi = c; }
+      }
+      c1 = bi;
+    }
+    chi[r] = c1;
+  }
+  __syncthreads();
+  APHASE(9);
+  if (tid < kKeys && j0 + tid < Nk && done) {
+    pidx[(size_t)bh * Nk + j0 + tid] = par[tid];
+    cidx[(size_t)bh * Nk + j0 + tid] = chi[tid];
+  }
+  APHASE(10);
 }
 
 uint32_t pow2_cols(int n) {
@@ -232,18 +307,25 @@ avq_status launch(const avq_problem& p, const void* K, const void* Cp, const voi
     avq_status s = make_tmap_bf16(&tmCp, Cp, 2, dims, box);
     if (s != AVQ_OK) return s;
   }
-  const size_t smem = 1024 + (size_t)(D / 64) * (kKeys + p.M) * 128 + sizeof(float) * p.M + 64;
+  const size_t smem = (size_t)(D / 64) * (kKeys + p.M) * 128 + sizeof(float) * (p.M + 6 * kKeys) +
+                      sizeof(int) * (4 * kKeys) + 64 + 1024;
   auto kern = tc_assign_kernel<D>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return AVQ_ERR_CUDA;
   dim3 grid((p.Nk + kKeys - 1) / kKeys, (unsigned)BH);
-  kern<<<grid, kKeys, smem, st>>>(tmK, tmCp, static_cast<const __nv_bfloat16*>(Cp),
-                                  static_cast<const __nv_bfloat16*>(Cc), pidx, cidx, p.H, p.Nk, p.M, p.C,
-                                  pow2_cols(p.M), status_word);
+  kern<<<grid, kThreadsA, smem, st>>>(tmK, tmCp, static_cast<const __nv_bfloat16*>(Cp),
+                                      static_cast<const __nv_bfloat16*>(Cc), pidx, cidx, p.H, p.Nk, p.M, p.C,
+                                      pow2_cols(p.M), status_word);
   return cuda_ok(cudaGetLastError());
 }
 
 }  // namespace
+
+#ifdef AVQ_PHASE_DEBUG
+extern "C" __attribute__((visibility("default"))) int avq_debug_assign_clocks(long long* host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, g_assign_clocks, sizeof(long long) * 64 * 16);
+}
+#endif
 
 avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const void* Cc,
                      int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, cudaStream_t st) {

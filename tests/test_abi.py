@@ -48,7 +48,7 @@ def test_workspace_bytes_and_layout(lib):
     offs = [ctypes.c_size_t() for _ in range(6)]
     assert lib.avq_workspace_layout(ctypes.byref(p), 2, 64, *[ctypes.byref(o) for o in offs]) == 0
     vals = [o.value for o in offs]
-    assert vals == sorted(vals) and vals[0] == 256 and all(v % 256 == 0 for v in vals)
+    assert len(set(vals)) == 6 and min(vals) == 256 and all(v % 256 == 0 for v in vals) and max(vals) < n
     pb = _prob(dtype_code=binding.AVQ_BF16, Nq=1024, Nk=1024, M=64)
     assert binding.workspace_bytes(pb, 8, 128) > binding.workspace_bytes(_prob(Nq=1024, Nk=1024, M=64), 8, 128)
 
