@@ -37,25 +37,28 @@ leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restri
     const int c = __ldg(cidx + kb + j0 + lane);
     leaf_l = a * C + c;
   }
-  using Vec = typename std::conditional<D == 128, uint2, uint32_t>::type;
-  Vec v[kKeysPerWarp];
+  // Every lane adds four floats with one 16-byte reduction: a full warp covers a 128-wide row, a
+  // half warp a 64-wide one (two keys per step).
+  constexpr int kLanesPerRow = D / 4;
+  constexpr int kRowsPerStep = 32 / kLanesPerRow;
+  constexpr int kSteps = kKeysPerWarp / kRowsPerStep;
+  const int sub = lane / kLanesPerRow, col = lane % kLanesPerRow;
+  uint2 v[kSteps];
 #pragma unroll
-  for (int t = 0; t < kKeysPerWarp; ++t)
-    if (j0 + t < Nk) v[t] = __ldg(reinterpret_cast<const Vec*>(V + (kb + j0 + t) * D) + lane);
+  for (int t = 0; t < kSteps; ++t) {
+    const int j = j0 + t * kRowsPerStep + sub;
+    v[t] = make_uint2(0u, 0u);
+    if (j < Nk) v[t] = __ldg(reinterpret_cast<const uint2*>(V + (kb + j) * D) + col);
+  }
 #pragma unroll
-  for (int t = 0; t < kKeysPerWarp; ++t) {
-    const int leaf = __shfl_sync(0xffffffffu, leaf_l, t);
-    if (leaf < 0) continue;                           // past the end (warp-uniform)
-    float* dst = Vc + ((size_t)bh * M * C + leaf) * D;
-    if constexpr (D == 128) {
+  for (int t = 0; t < kSteps; ++t) {
+    const int leaf = __shfl_sync(0xffffffffu, leaf_l, t * kRowsPerStep + sub);
+    if (leaf >= 0) {
+      float* dst = Vc + ((size_t)bh * M * C + leaf) * D;
       const uint2 u = v[t];
-      atomicAdd(reinterpret_cast<float4*>(dst) + lane,
+      atomicAdd(reinterpret_cast<float4*>(dst) + col,
                 make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u),
                             __uint_as_float(u.y << 16), __uint_as_float(u.y & 0xFFFF0000u)));
-    } else {
-      const uint32_t u = v[t];
-      atomicAdd(reinterpret_cast<float2*>(dst) + lane,
-                make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u)));
     }
   }
   if (leaf_l >= 0) atomicAdd(nc + (size_t)bh * M * C + leaf_l, 1.0f);

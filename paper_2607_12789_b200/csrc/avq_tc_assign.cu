@@ -7,9 +7,11 @@
 //            the best and the runner-up; the halves are merged in shared memory.  Only when best and
 //            runner-up are closer than the MMA's rounding can separate are all M distances redone in
 //            float64 in the direct form (lowest index wins ties).
-//   child    the two threads of a key split the C children of its parent and evaluate the direct form
-//            sum (k - c)^2 in fp32 on CUDA cores (2 C d flops per key; a second MMA over all M C
-//            children would cost C times the parent GEMM).  Same float64 recheck for near-ties.
+//   child    fp32 direct form sum (k - c)^2 on CUDA cores (2 C d flops per key; a second MMA over all
+//            M C children would cost C times the parent GEMM), float64 recheck for near-ties.  Small
+//            child blocks (C d = 256): the two threads of a key take half of the children each.
+//            Larger ones: a warp fetches a key's contiguous C x d block with coalesced 16-byte loads,
+//            every lane squares its 8 differences and shuffles reduce per child.
 #include "avq_tc_common.cuh"
 
 namespace avq {
@@ -62,7 +64,8 @@ __device__ double exact_dist_smem(const unsigned char* Ks, int row, const __nv_b
   return s;
 }
 
-template <int D>
+// NL = 16-byte loads per lane that cover one parent's C x d block of children: C * d / 256.
+template <int D, int NL>
 __global__ void __launch_bounds__(kThreadsA, 2)
 tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmCp,
                  const __nv_bfloat16* __restrict__ Cp, const __nv_bfloat16* __restrict__ Cc,
@@ -228,52 +231,127 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   __syncthreads();
   APHASE(8);
 
-  // ---- child argmin: the two threads of a key take half of the C children each (fp32 direct form),
-  // eight 16-byte loads in flight per thread; the halves are merged like the parents'
-  {
-    const int a = par[r];
-    const int CH = C >> 1;                           // children per thread (C is 4 or 8)
-    const __nv_bfloat16* Cch = Cc + (((size_t)h * M + a) * C + (size_t)hf * CH) * D;
-    float e1 = INFINITY, e2 = INFINITY;
-    int c1 = 0;
-    for (int c = 0; c < CH; ++c) {
-      const uint4* src = reinterpret_cast<const uint4*>(Cch + (size_t)c * D);
-      float s = 0.f;
-#pragma unroll
-      for (int g = 0; g < D / 64; ++g) {             // 8 chunks (64 elements) at a time
-        uint4 cv[8];
-#pragma unroll
-        for (int t = 0; t < 8; ++t) cv[t] = __ldg(src + g * 8 + t);
-#pragma unroll
-        for (int t = 0; t < 8; ++t) {
-          const uint4 kv = *reinterpret_cast<const uint4*>(Ks + g * kKeys * 128 + sw128_offset(r, t * 8));
-          s += sqdiff8(kv, cv[t]);
+  if constexpr (NL == 1) {
+    // ---- child argmin: the two threads of a key take half of the C children each (fp32 direct form),
+    // eight 16-byte loads in flight per thread; the halves are merged like the parents'
+    {
+      const int a = par[r];
+      const int CH = C >> 1;                           // children per thread (C is 4 or 8)
+      const __nv_bfloat16* Cch = Cc + (((size_t)h * M + a) * C + (size_t)hf * CH) * D;
+      float e1 = INFINITY, e2 = INFINITY;
+      int c1 = 0;
+      for (int c = 0; c < CH; ++c) {
+        const uint4* src = reinterpret_cast<const uint4*>(Cch + (size_t)c * D);
+        float s = 0.f;
+  #pragma unroll
+        for (int g = 0; g < D / 64; ++g) {             // 8 chunks (64 elements) at a time
+          uint4 cv[8];
+  #pragma unroll
+          for (int t = 0; t < 8; ++t) cv[t] = __ldg(src + g * 8 + t);
+  #pragma unroll
+          for (int t = 0; t < 8; ++t) {
+            const uint4 kv = *reinterpret_cast<const uint4*>(Ks + g * kKeys * 128 + sw128_offset(r, t * 8));
+            s += sqdiff8(kv, cv[t]);
+          }
         }
+        e2 = fminf(e2, fmaxf(s, e1));
+        if (s < e1) { e1 = s; c1 = hf * CH + c; }
       }
-      e2 = fminf(e2, fmaxf(s, e1));
-      if (s < e1) { e1 = s; c1 = hf * CH + c; }
+      xd1[hf * kKeys + r] = e1;
+      xd2[hf * kKeys + r] = e2;
+      xi1[hf * kKeys + r] = c1;
     }
-    xd1[hf * kKeys + r] = e1;
-    xd2[hf * kKeys + r] = e2;
-    xi1[hf * kKeys + r] = c1;
-  }
-  __syncthreads();
-  if (hf == 0) {
-    const float a1 = xd1[r], a2 = xd2[r], b1 = xd1[kKeys + r], b2 = xd2[kKeys + r];
-    int c1 = (b1 < a1) ? xi1[kKeys + r] : xi1[r];
-    const float e1 = fminf(a1, b1);
-    const float e2 = fminf(fmaxf(a1, b1), fminf(a2, b2));
-    if (done && j0 + r < Nk && !(e2 - e1 > 1e-4f * e2)) {
-      const __nv_bfloat16* Cch = Cc + ((size_t)h * M + par[r]) * C * D;
-      double best = INFINITY;
-      int bi = 0;
-      for (int c = 0; c < C; ++c) {
-        const double s = exact_dist_smem<D>(Ks, r, Cch + (size_t)c * D);
-        if (s < best) { best = s; bi = c; }
+    __syncthreads();
+    if (hf == 0) {
+      const float a1 = xd1[r], a2 = xd2[r], b1 = xd1[kKeys + r], b2 = xd2[kKeys + r];
+      int c1 = (b1 < a1) ? xi1[kKeys + r] : xi1[r];
+      const float e1 = fminf(a1, b1);
+      const float e2 = fminf(fmaxf(a1, b1), fminf(a2, b2));
+      if (done && j0 + r < Nk && !(e2 - e1 > 1e-4f * e2)) {
+        const __nv_bfloat16* Cch = Cc + ((size_t)h * M + par[r]) * C * D;
+        double best = INFINITY;
+        int bi = 0;
+        for (int c = 0; c < C; ++c) {
+          const double s = exact_dist_smem<D>(Ks, r, Cch + (size_t)c * D);
+          if (s < best) { best = s; bi = c; }
+        }
+        c1 = bi;
       }
-      c1 = bi;
+      chi[r] = c1;
     }
-    chi[r] = c1;
+  } else {
+    // ---- child argmin, one warp per key (16 keys per warp).  A parent's C children are one contiguous
+    // C x d block: NL fully coalesced 16-byte loads per lane fetch it.  Lane l holds 8 elements of child
+    // (t * kChildPerLoad + l / kLanesPerChild) for load t; it squares its 8 differences against the key row,
+    // a butterfly sums them per child, a second butterfly merges (best, index, runner-up) over children.
+    // Loads of the next batch of keys are in flight while the current batch is reduced.
+    {
+      constexpr int kLanesPerChild = D / 8;
+      constexpr int kChildPerLoad = 32 / kLanesPerChild;
+      constexpr int kKB = (NL >= 4) ? 1 : 4 / NL;      // keys per batch: 4 loads per lane in flight per buffer
+      constexpr int kNB = 16 / kKB;                    // batches per warp
+      const int kpos = (lane % kLanesPerChild) * 8;    // first key element this lane compares
+      const int grp = lane / kLanesPerChild;
+      const unsigned char* krow_base = Ks + (kpos >> 6) * (kKeys * 128);
+      const size_t head_base = (size_t)h * M;
+      uint4 buf[2][kKB][NL];
+      auto issue = [&](int bsel, int batch) {
+  #pragma unroll
+        for (int b = 0; b < kKB; ++b) {
+          const int key = warp * 16 + batch * kKB + b;
+          const uint4* src = reinterpret_cast<const uint4*>(Cc + (head_base + par[key]) * C * D) + lane;
+  #pragma unroll
+          for (int t = 0; t < NL; ++t) buf[bsel][b][t] = __ldg(src + t * 32);
+        }
+      };
+      auto reduce = [&](int bsel, int batch) {
+  #pragma unroll
+        for (int b = 0; b < kKB; ++b) {
+          const int key = warp * 16 + batch * kKB + b;
+          const uint4 kv = *reinterpret_cast<const uint4*>(krow_base + sw128_offset(key, kpos & 63));
+          float e1 = INFINITY, e2 = INFINITY;
+          int c1 = 0;
+  #pragma unroll
+          for (int t = 0; t < NL; ++t) {
+            float s = sqdiff8(kv, buf[bsel][b][t]);
+  #pragma unroll
+            for (int o = 1; o < kLanesPerChild; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            const int c = t * kChildPerLoad + grp;     // ascending in t: a later equal distance never wins
+            e2 = fminf(e2, fmaxf(s, e1));
+            if (s < e1) { e1 = s; c1 = c; }
+          }
+  #pragma unroll
+          for (int o = kLanesPerChild; o < 32; o <<= 1) {
+            const float b1 = __shfl_xor_sync(0xffffffffu, e1, o);
+            const float b2 = __shfl_xor_sync(0xffffffffu, e2, o);
+            const int cb = __shfl_xor_sync(0xffffffffu, c1, o);
+            e2 = fminf(fmaxf(e1, b1), fminf(e2, b2));
+            if (b1 < e1 || (b1 == e1 && cb < c1)) { e1 = b1; c1 = cb; }
+          }
+          if (lane == 0) {
+            if (done && j0 + key < Nk && C > 1 && !(e2 - e1 > 1e-4f * e2)) {
+              const __nv_bfloat16* Cch = Cc + (head_base + par[key]) * C * D;
+              double best = INFINITY;
+              int bi = 0;
+              for (int c = 0; c < C; ++c) {
+                const double sd = exact_dist_smem<D>(Ks, key, Cch + (size_t)c * D);
+                if (sd < best) { best = sd; bi = c; }
+              }
+              c1 = bi;
+            }
+            chi[key] = c1;
+          }
+        }
+      };
+      issue(0, 0);
+  #pragma unroll
+      for (int batch = 0; batch < kNB; batch += 2) {
+        issue(1, batch + 1);
+        reduce(0, batch);
+        if (batch + 2 < kNB) issue(0, batch + 2);
+        reduce(1, batch + 1);
+      }
+    }
   }
   __syncthreads();
   APHASE(9);
@@ -290,7 +368,7 @@ uint32_t pow2_cols(int n) {
   return c;
 }
 
-template <int D>
+template <int D, int NL>
 avq_status launch(const avq_problem& p, const void* K, const void* Cp, const void* Cc, int32_t* pidx,
                   int32_t* cidx, int32_t* status_word, cudaStream_t st) {
   CUtensorMap tmK, tmCp;
@@ -309,7 +387,7 @@ avq_status launch(const avq_problem& p, const void* K, const void* Cp, const voi
   }
   const size_t smem = (size_t)(D / 64) * (kKeys + p.M) * 128 + sizeof(float) * (p.M + 6 * kKeys) +
                       sizeof(int) * (4 * kKeys) + 64 + 1024;
-  auto kern = tc_assign_kernel<D>;
+  auto kern = tc_assign_kernel<D, NL>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return AVQ_ERR_CUDA;
   dim3 grid((p.Nk + kKeys - 1) / kKeys, (unsigned)BH);
@@ -329,8 +407,11 @@ extern "C" __attribute__((visibility("default"))) int avq_debug_assign_clocks(lo
 
 avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const void* Cc,
                      int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, cudaStream_t st) {
-  return p.d == 64 ? launch<64>(p, K, Cp, Cc, parent_idx, child_idx, status_word, st)
-                   : launch<128>(p, K, Cp, Cc, parent_idx, child_idx, status_word, st);
+  if (p.d == 64)
+    return p.C == 4 ? launch<64, 1>(p, K, Cp, Cc, parent_idx, child_idx, status_word, st)
+                    : launch<64, 2>(p, K, Cp, Cc, parent_idx, child_idx, status_word, st);
+  return p.C == 4 ? launch<128, 2>(p, K, Cp, Cc, parent_idx, child_idx, status_word, st)
+                  : launch<128, 4>(p, K, Cp, Cc, parent_idx, child_idx, status_word, st);
 }
 
 }  // namespace avq

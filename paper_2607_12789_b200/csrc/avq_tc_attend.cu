@@ -117,7 +117,8 @@ __device__ __forceinline__ float store_weights16(unsigned char* A, int r, int co
 template <int D, int NQ, int CT>
 __global__ void __launch_bounds__(128 * NQ, 4 / NQ)
 tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmCp,
-                 const __grid_constant__ CUtensorMap tmVpT, const AttendParams p) {
+                 const __grid_constant__ CUtensorMap tmVpT, const __grid_constant__ CUtensorMap tmY,
+                 const AttendParams p) {
   // 1024-byte alignment (swizzle atoms) is requested from the launch, not computed from the pointer, so
   // that the compiler keeps every access in the shared address space.
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -162,10 +163,9 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   uint64_t* bar_pv = &bars[3];
 
   // A wait that expired in an earlier CTA of this launch: do not start more work.
+  // The flag is read here and acted on after the set-up barrier below, so that it costs no extra round trip.
   __shared__ int early_exit;
   if (tid == 0) early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
-  __syncthreads();
-  if (early_exit) return;
   PHASE_MARK(0);
 
   // ---- barriers, then the loads first: Q tile + parent codebook, and the parents' value sums
@@ -200,6 +200,14 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (early_exit) {
+    // let the loads already in flight land in this CTA's shared memory, then leave cleanly
+    mbar_wait(bar_ld0, 0, abort_flag, nullptr, 0);
+    mbar_wait(bar_ld1, 0, abort_flag, nullptr, 0);
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+    return;
+  }
   const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
   const uint32_t t_s = t_row + (uint32_t)colbase;
   const uint32_t t_sc = t_row + (uint32_t)(cq * QWC);
@@ -588,24 +596,30 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tc_fence_after();
   PHASE_MARK(27);
   if (o_ok) {
-    // tcgen05.ld is warp-collective: every lane loads, only rows inside the tensor store.
+    // The output tile is staged in shared memory (over the Q tile, which no MMA reads any more) in the
+    // layout of the Q load and written with TMA tile stores; rows past Nq are clipped by the tensor map.
     const float inv = 1.f / z_run;
-    __nv_bfloat16* yrow = p.Y + ((size_t)bh * p.Nq + i0 + r) * D + cq * (D / NQ);
     for (int c0 = 0; c0 < D / NQ; c0 += 16) {
       float o[16];
       tmem_ld16(t_o + c0, o);
       uint32_t pk[8];
 #pragma unroll
       for (int e = 0; e < 16; e += 2) pk[e >> 1] = pack_bf16(o[e] * inv, o[e + 1] * inv);
-      if (r < rows_valid) {
-        *reinterpret_cast<uint4*>(yrow + c0) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-        *reinterpret_cast<uint4*>(yrow + c0 + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-      }
+      const int col0 = cq * (D / NQ) + c0;
+      unsigned char* sub = Qs + (col0 >> 6) * (kRows * 128);
+      *reinterpret_cast<uint4*>(sub + sw128_offset(r, col0 & 63)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      *reinterpret_cast<uint4*>(sub + sw128_offset(r, (col0 & 63) + 8)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
     }
+    fence_proxy_async();
   }
-  PHASE_MARK(28);
   tc_fence_before();
   __syncthreads();
+  if (tid == 0 && o_ok) {
+#pragma unroll
+    for (int s2 = 0; s2 < kSubD; ++s2) tma_store_3d(&tmY, Qs + s2 * kRows * 128, s2 * 64, i0, bh);
+    tma_store_commit_and_wait_read();
+  }
+  PHASE_MARK(28);
   if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
   PHASE_MARK(29);
 }
@@ -621,12 +635,12 @@ size_t attend_smem(int D, int CT, int CHW) {
 
 template <int D, int NQ, int CT>
 avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUtensorMap& tmVpT,
-                     const AttendParams& a, unsigned BH, size_t smem, cudaStream_t st) {
+                     const CUtensorMap& tmY, const AttendParams& a, unsigned BH, size_t smem, cudaStream_t st) {
   auto kern = tc_attend_kernel<D, NQ, CT>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return AVQ_ERR_CUDA;
   dim3 grid(a.nblk, BH);
-  kern<<<grid, 128 * NQ, smem, st>>>(tmQ, tmCp, tmVpT, a);
+  kern<<<grid, 128 * NQ, smem, st>>>(tmQ, tmCp, tmVpT, tmY, a);
   return cuda_ok(cudaGetLastError());
 }
 
@@ -635,11 +649,13 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
                   const float* nc, const void* VpT, const void* VcT, int32_t P, void* Y, int32_t* topp_out,
                   float* importance_out, int32_t* status_word, cudaStream_t st) {
   const uint64_t BH = (uint64_t)p.B * p.H;
-  CUtensorMap tmQ, tmCp, tmVpT;
+  CUtensorMap tmQ, tmCp, tmVpT, tmY;
   {
     const uint64_t dims[3] = {(uint64_t)D, (uint64_t)p.Nq, BH};
     const uint32_t box[3] = {64, (uint32_t)kRows, 1};
     avq_status s = make_tmap_bf16(&tmQ, Q, 3, dims, box);
+    if (s != AVQ_OK) return s;
+    s = make_tmap_bf16(&tmY, Y, 3, dims, box);
     if (s != AVQ_OK) return s;
   }
   {
@@ -677,13 +693,13 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
   // four small CTAs of 128 threads, two of 256, or one of 512.
   const unsigned bh = (unsigned)BH;
   if (D == 64) {
-    if (CT == 64) return launch_nq<D, 1, 64>(tmQ, tmCp, tmVpT, a, bh, smem, st);
-    if (CT == 128) return launch_nq<D, 2, 128>(tmQ, tmCp, tmVpT, a, bh, smem, st);
-    return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, a, bh, smem, st);
+    if (CT == 64) return launch_nq<D, 1, 64>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
+    if (CT == 128) return launch_nq<D, 2, 128>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
+    return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
   }
-  if (CT == 64) return launch_nq<D, 2, 64>(tmQ, tmCp, tmVpT, a, bh, smem, st);
-  if (CT == 128) return launch_nq<D, 4, 128>(tmQ, tmCp, tmVpT, a, bh, smem, st);
-  return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, a, bh, smem, st);
+  if (CT == 64) return launch_nq<D, 2, 64>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
+  if (CT == 128) return launch_nq<D, 4, 128>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
+  return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
 }
 
 }  // namespace
