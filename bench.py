@@ -279,6 +279,8 @@ def main():
     ap.add_argument("--workload", default="c1")
     ap.add_argument("--also", default="c2,c3", help="comma list of further workloads reported under 'also'")
     ap.add_argument("--simt", action="store_true", help="force the CUDA-core kernels (cross-check)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time every (N, M, P) point of the sweep configuration; one JSON line per point")
     ap.add_argument("--profile", action="store_true",
                     help="only W warm-up and K timed steps (no stage timing, e2e, CPU baseline): for ncu")
     args = ap.parse_args()
@@ -320,6 +322,20 @@ def main():
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
     flags = 2 if args.simt else 0
     pk = peaks()
+    if args.sweep:
+        from paper_2607_12789_b200 import synth
+        for N in synth.SWEEP_N:
+            for M in synth.SWEEP_M:
+                for P in synth.sweep_P(M):
+                    w2 = synth.sweep_point(N, M, P)
+                    r2 = run_gpu(w2, max(5, args.steps // 5), 3, 0, 1, flags=flags, extras=False, min_warm_s=0.0)
+                    _, f2 = model(w2)
+                    fr2 = roof(f2, pk, r2["ms"], w2.dtype)
+                    print(json.dumps(dict(workload=w2.name, N=N, M=M, P=P, ms_per_step=r2["ms"],
+                                          value=w2.B * w2.N / (r2["ms"] * 1e-3), unit=UNIT,
+                                          tflops=f2["flops"] / (r2["ms"] * 1e-3) / 1e12, bound=fr2["bound"],
+                                          forward_roofline_frac=fr2["frac"])), flush=True)
+        return
     if args.profile:
         res = run_gpu(wl, args.steps, warm, rank, world, flags=flags, extras=False, min_warm_s=0.0)
         if rank == 0:

@@ -97,6 +97,8 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
   APHASE(0);
   if (tid == 0) {
+    prefetch_tmap(&tmK);
+    prefetch_tmap(&tmCp);
     mbar_init(&bars[0], 1);
     mbar_init(&bars[1], 1);
     mbar_fence_init();

@@ -142,10 +142,10 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   float* biasc = cntc + CHW;                             // [CHW]
   float* w = biasc + CHW;                                // [256] importance
   float* wpart = w + 256;                                // [4][CT]
-  float* xm = wpart + 4 * CT;                            // [4][128] exchange between the threads of a row
-  float* xz = xm + 4 * kRows;                            // [4][128]
-  float* xz2 = xz + 4 * kRows;                           // [4][128]
-  int* sel_list = reinterpret_cast<int*>(xz2 + 4 * kRows);   // [256]
+  float* xm = wpart + 4 * CT;                            // [NQ][128] exchange between the threads of a row
+  float* xz = xm + NQ * kRows;                           // [NQ][128]
+  float* xz2 = xz + NQ * kRows;                          // [NQ][128]
+  int* sel_list = reinterpret_cast<int*>(xz2 + NQ * kRows);   // [256]
   uint32_t* wmask = reinterpret_cast<uint32_t*>(sel_list + 256);   // [16]
   uint64_t* bars = reinterpret_cast<uint64_t*>(wmask + 18);        // [4]  (wmask[16] is a scratch word)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4);
@@ -170,6 +170,9 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
   // ---- barriers, then the loads first: Q tile + parent codebook, and the parents' value sums
   if (tid == 0) {
+    prefetch_tmap(&tmQ);
+    prefetch_tmap(&tmCp);
+    prefetch_tmap(&tmVpT);
     mbar_init(bar_ld0, 1);
     mbar_init(bar_ld1, 1);
     mbar_init(bar_s, 1);
@@ -332,8 +335,8 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // that when a group of EQUAL importances straddles the boundary only its lowest indices are kept.
   // kT threads share one parent's scan.
   {
-    constexpr int kT = NQ >= 2 ? 2 : 1;                  // 128 * NQ >= kT * M for every launch shape
-    const int j = tid / kT, part = tid % kT;
+    const int kT = (kThreads >= 2 * M) ? 2 : 1;          // threads that share one parent's scan
+    const int j = (kT == 2) ? (tid >> 1) : tid, part = (kT == 2) ? (tid & 1) : 0;
     const uint32_t* keys = reinterpret_cast<const uint32_t*>(w);
     int* gstar = reinterpret_cast<int*>(&wmask[16]);
     bool mine = false;
@@ -624,11 +627,11 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   PHASE_MARK(29);
 }
 
-size_t attend_smem(int D, int CT, int CHW) {
+size_t attend_smem(int D, int CT, int CHW, int NQ) {
   const int subA = CT / 64;
   const size_t ca = (size_t)max(CT * D * 2, subA * kRows * 128);
-  size_t b = 1024 + (size_t)(D / 64) * kRows * 128 + ca + (size_t)subA * D * 128 + (size_t)CHW * D * 2;
-  b += sizeof(float) * (3 * (size_t)CT + 2 * (size_t)CHW + 256 + 4 * (size_t)CT + 12 * kRows);
+  size_t b = (size_t)(D / 64) * kRows * 128 + ca + (size_t)subA * D * 128 + (size_t)CHW * D * 2;
+  b += sizeof(float) * (3 * (size_t)CT + 2 * (size_t)CHW + 256 + 4 * (size_t)CT + 3 * (size_t)NQ * kRows);
   b += sizeof(int) * 256 + sizeof(uint32_t) * 18 + sizeof(uint64_t) * 4 + 2 * sizeof(uint32_t);
   return b + 64;
 }
@@ -688,7 +691,8 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
   while ((int)cols < CT + D) cols <<= 1;
   a.tmem_cols = cols;
   a.scale_log2e = p.scale * 1.4426950408889634f;
-  const size_t smem = attend_smem(D, CT, CHW);
+  const int NQ = (D == 64) ? (CT == 64 ? 1 : (CT == 128 ? 2 : 4)) : (CT == 64 ? 2 : 4);
+  const size_t smem = attend_smem(D, CT, CHW, NQ);
   // Threads per query row follow from how many CTAs can share an SM (TMEM columns, shared memory):
   // four small CTAs of 128 threads, two of 256, or one of 512.
   const unsigned bh = (unsigned)BH;
