@@ -68,6 +68,7 @@ __device__ double exact_dist_smem(const unsigned char* Ks, int row, const __nv_b
 template <int D, int NL>
 __global__ void __launch_bounds__(kThreadsA, 2)
 tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmCp,
+                 const __grid_constant__ CUtensorMap tmCc, const int stage_rows_arg,
                  const __nv_bfloat16* __restrict__ Cp, const __nv_bfloat16* __restrict__ Cc,
                  int32_t* __restrict__ pidx, int32_t* __restrict__ cidx, int H, int Nk, int M, int C,
                  uint32_t tmem_cols, int32_t* status_word) {
@@ -77,7 +78,11 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   constexpr int kSub = D / 64;                       // 64-column sub-tiles along the head dimension
   unsigned char* Ks = smem;                          // kSub x [128 x 128 B]
   unsigned char* Cs = Ks + kSub * kKeys * 128;       // kSub x [M x 128 B]
-  float* cnorm = reinterpret_cast<float*>(Cs + kSub * M * 128);   // [M]
+  const int stage_rows = (NL == 1) ? stage_rows_arg : 0;   // only the small-block variant stages
+  // Small child codebooks (stage_rows = M * C rows of 128 bytes, d = 64 only) are staged whole, so that
+  // the child argmin reads shared memory instead of gathering rows from global memory.
+  unsigned char* Ccs = Cs + kSub * M * 128;          // [stage_rows x 128 B], 128-byte swizzle
+  float* cnorm = reinterpret_cast<float*>(Ccs + stage_rows * 128);   // [M]
   float* xd1 = cnorm + M;                            // [2][128] best distance of each column half
   float* xd2 = xd1 + 2 * kKeys;                      // [2][128] runner-up
   float* xkn = xd2 + 2 * kKeys;                      // [2][128] halves of ||k||^2
@@ -99,12 +104,15 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   if (tid == 0) {
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmCp);
+    if (stage_rows) prefetch_tmap(&tmCc);
     mbar_init(&bars[0], 1);
     mbar_init(&bars[1], 1);
     mbar_fence_init();
     *abort_flag = 0;
     *cmax_bits = 0;
-    mbar_expect_tx(&bars[0], (uint32_t)(kSub * (kKeys + M) * 128));
+    mbar_expect_tx(&bars[0], (uint32_t)(kSub * (kKeys + M) * 128 + stage_rows * 128));
+    for (int b0 = 0; b0 < stage_rows; b0 += 256)
+      tma_load_2d(Ccs + b0 * 128, &tmCc, 0, h * M * C + b0, &bars[0]);
 #pragma unroll
     for (int s = 0; s < kSub; ++s) {
       tma_load_3d(Ks + s * kKeys * 128, &tmK, s * 64, j0, bh, &bars[0]);
@@ -249,7 +257,9 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         for (int g = 0; g < D / 64; ++g) {             // 8 chunks (64 elements) at a time
           uint4 cv[8];
   #pragma unroll
-          for (int t = 0; t < 8; ++t) cv[t] = __ldg(src + g * 8 + t);
+          for (int t = 0; t < 8; ++t)
+            cv[t] = stage_rows ? *reinterpret_cast<const uint4*>(Ccs + sw128_offset(a * C + hf * CH + c, t * 8))
+                               : __ldg(src + g * 8 + t);
   #pragma unroll
           for (int t = 0; t < 8; ++t) {
             const uint4 kv = *reinterpret_cast<const uint4*>(Ks + g * kKeys * 128 + sw128_offset(r, t * 8));
@@ -373,8 +383,16 @@ uint32_t pow2_cols(int n) {
 template <int D, int NL>
 avq_status launch(const avq_problem& p, const void* K, const void* Cp, const void* Cc, int32_t* pidx,
                   int32_t* cidx, int32_t* status_word, cudaStream_t st) {
-  CUtensorMap tmK, tmCp;
+  CUtensorMap tmK, tmCp, tmCc;
   const uint64_t BH = (uint64_t)p.B * p.H;
+  // stage the head's whole child codebook when it is small (d = 64, C = 4, at most 512 rows = 64 KB)
+  const int stage_rows = (NL == 1 && p.M * p.C <= 512) ? p.M * p.C : 0;
+  {
+    const uint64_t dims[2] = {(uint64_t)D, (uint64_t)p.H * p.M * p.C};
+    const uint32_t box[2] = {64, (uint32_t)(stage_rows > 256 ? 256 : (stage_rows ? stage_rows : 8))};
+    avq_status s = make_tmap_bf16(&tmCc, Cc, 2, dims, box);
+    if (s != AVQ_OK) return s;
+  }
   {
     const uint64_t dims[3] = {(uint64_t)D, (uint64_t)p.Nk, BH};
     const uint32_t box[3] = {64, (uint32_t)kKeys, 1};
@@ -387,13 +405,21 @@ avq_status launch(const avq_problem& p, const void* K, const void* Cp, const voi
     avq_status s = make_tmap_bf16(&tmCp, Cp, 2, dims, box);
     if (s != AVQ_OK) return s;
   }
-  const size_t smem = (size_t)(D / 64) * (kKeys + p.M) * 128 + sizeof(float) * (p.M + 6 * kKeys) +
+  const size_t smem = (size_t)(D / 64) * (kKeys + p.M) * 128 + (size_t)stage_rows * 128 +
+                      sizeof(float) * (p.M + 6 * kKeys) +
                       sizeof(int) * (4 * kKeys) + 64 + 1024;
   auto kern = tc_assign_kernel<D, NL>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return AVQ_ERR_CUDA;
+  // The limit is set once per device and instantiation (setting it again is harmless if two threads race).
+  static size_t configured[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return AVQ_ERR_CUDA;
+  if (dev < 0 || dev >= 64 || smem > configured[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return AVQ_ERR_CUDA;
+    if (dev >= 0 && dev < 64) configured[dev] = smem;
+  }
   dim3 grid((p.Nk + kKeys - 1) / kKeys, (unsigned)BH);
-  kern<<<grid, kThreadsA, smem, st>>>(tmK, tmCp, static_cast<const __nv_bfloat16*>(Cp),
+  kern<<<grid, kThreadsA, smem, st>>>(tmK, tmCp, tmCc, stage_rows, static_cast<const __nv_bfloat16*>(Cp),
                                       static_cast<const __nv_bfloat16*>(Cc), pidx, cidx, p.H, p.Nk, p.M, p.C,
                                       pow2_cols(p.M), status_word);
   return cuda_ok(cudaGetLastError());

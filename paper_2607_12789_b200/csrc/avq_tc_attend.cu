@@ -640,8 +640,15 @@ template <int D, int NQ, int CT>
 avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUtensorMap& tmVpT,
                      const CUtensorMap& tmY, const AttendParams& a, unsigned BH, size_t smem, cudaStream_t st) {
   auto kern = tc_attend_kernel<D, NQ, CT>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return AVQ_ERR_CUDA;
+  // The limit is set once per device and instantiation (setting it again is harmless if two threads race).
+  static size_t configured[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return AVQ_ERR_CUDA;
+  if (dev < 0 || dev >= 64 || smem > configured[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return AVQ_ERR_CUDA;
+    if (dev >= 0 && dev < 64) configured[dev] = smem;
+  }
   dim3 grid(a.nblk, BH);
   kern<<<grid, 128 * NQ, smem, st>>>(tmQ, tmCp, tmVpT, tmY, a);
   return cuda_ok(cudaGetLastError());
