@@ -33,19 +33,34 @@ __device__ long long g_assign_clocks[64 * 16];
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
 
-// sum over 8 bf16 pairs of (a - b)^2 for two packed 16-byte chunks
-__device__ __forceinline__ float sqdiff8(const uint4& a, const uint4& b) {
-  const uint32_t x[4] = {a.x, a.y, a.z, a.w}, y[4] = {b.x, b.y, b.z, b.w};
-  float s = 0.f;
+// Two packed bf16 widened to a pair of fp32 in one 64-bit register (for the f32x2 instructions).
+__device__ __forceinline__ uint64_t bf2_to_f32x2(uint32_t u) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(u << 16), "r"(u & 0xFFFF0000u));
+  return r;
+}
+struct KeyChunk { uint64_t p[4]; };   // 8 key elements as four fp32 pairs
+__device__ __forceinline__ KeyChunk widen8(const uint4& a) {
+  KeyChunk k;
+  k.p[0] = bf2_to_f32x2(a.x); k.p[1] = bf2_to_f32x2(a.y); k.p[2] = bf2_to_f32x2(a.z); k.p[3] = bf2_to_f32x2(a.w);
+  return k;
+}
+// sum over 8 elements of (k - c)^2, two lanes of packed fp32 arithmetic (sub.f32x2 / fma.f32x2)
+__device__ __forceinline__ float sqdiff8(const KeyChunk& k, const uint4& c) {
+  const uint32_t y[4] = {c.x, c.y, c.z, c.w};
+  uint64_t acc = 0;   // {0.f, 0.f}
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
-    const float d0 = bf_lo(x[e]) - bf_lo(y[e]);
-    const float d1 = bf_hi(x[e]) - bf_hi(y[e]);
-    s = fmaf(d0, d0, s);
-    s = fmaf(d1, d1, s);
+    uint64_t d;
+    const uint64_t cw = bf2_to_f32x2(y[e]);
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(k.p[e]), "l"(cw));
+    asm("fma.rn.f32x2 %0, %1, %1, %0;" : "+l"(acc) : "l"(d));
   }
-  return s;
+  float lo, hi;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(acc));
+  return lo + hi;
 }
+__device__ __forceinline__ float sqdiff8(const uint4& a, const uint4& b) { return sqdiff8(widen8(a), b); }
 
 // element `col` (0..D-1) of key row `row` in the swizzled key tile
 template <int D>
@@ -66,7 +81,7 @@ __device__ double exact_dist_smem(const unsigned char* Ks, int row, const __nv_b
 
 // NL = 16-byte loads per lane that cover one parent's C x d block of children: C * d / 256.
 template <int D, int NL>
-__global__ void __launch_bounds__(kThreadsA, 2)
+__global__ void __launch_bounds__(kThreadsA, NL == 1 ? 3 : 2)
 tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmCp,
                  const __grid_constant__ CUtensorMap tmCc, const int stage_rows_arg,
                  const __nv_bfloat16* __restrict__ Cp, const __nv_bfloat16* __restrict__ Cc,
@@ -320,7 +335,7 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   #pragma unroll
         for (int b = 0; b < kKB; ++b) {
           const int key = warp * 16 + batch * kKB + b;
-          const uint4 kv = *reinterpret_cast<const uint4*>(krow_base + sw128_offset(key, kpos & 63));
+          const KeyChunk kv = widen8(*reinterpret_cast<const uint4*>(krow_base + sw128_offset(key, kpos & 63)));
           float e1 = INFINITY, e2 = INFINITY;
           int c1 = 0;
   #pragma unroll
