@@ -3,8 +3,8 @@
 // One CTA = one query tile of 128 rows of one (batch, head); each row is handled by NQ threads
 // (column slices).  Flow of a tile:
 //   parents   S = Q . Cp^T                 tcgen05.mma, fp32 accumulator in TMEM columns [0, M)
-//             row maximum over non-empty parents, exp2, weights parked in TMEM as fp32,
-//             exact denominator z                                   (Eq. "vqflashattention")
+//             read once into registers: row maximum over non-empty parents, exp2, exact
+//             denominator z                                         (Eq. "vqflashattention")
 //             importance w_j = n_j sum_i A_ij / z_i from the fp32 weights  (Eq. "importance")
 //             top-P by rank, ties to the lower index                ("Child spawning")
 //             bf16 weights with the selected parents' columns zeroed -> shared memory
@@ -242,81 +242,95 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   ph_s ^= 1;
   tc_fence_after();
   PHASE_MARK(3);
+  // This thread's QW (<= 64) parent logits are read from TMEM once and stay in registers through the
+  // maximum, the exponentials, the importance sums and the conversion to bf16.
+  float a[QW];
   float mx = -INFINITY;
-  for (int c0 = 0; c0 < my_cols; c0 += 16) {
-    float s[16];
-    tmem_ld16(t_s + c0, s);
-    const float4* b4 = reinterpret_cast<const float4*>(bias + colbase + c0);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const float4 b = b4[u];
-      mx = fmaxf(mx, fmaxf(s[4 * u] + b.x, s[4 * u + 1] + b.y));
-      mx = fmaxf(mx, fmaxf(s[4 * u + 2] + b.z, s[4 * u + 3] + b.w));
+  for (int c0 = 0; c0 < QW; c0 += 16) {
+    if (c0 < my_cols) {                                  // warp-uniform
+      float s[16];
+      tmem_ld16(t_s + c0, s);
+      const float4* b4 = reinterpret_cast<const float4*>(bias + colbase + c0);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float4 b = b4[u];
+        mx = fmaxf(mx, fmaxf(s[4 * u] + b.x, s[4 * u + 1] + b.y));
+        mx = fmaxf(mx, fmaxf(s[4 * u + 2] + b.z, s[4 * u + 3] + b.w));
+      }
+#pragma unroll
+      for (int e = 0; e < 16; ++e) a[c0 + e] = s[e];
+    } else {
+#pragma unroll
+      for (int e = 0; e < 16; ++e) a[c0 + e] = 0.f;
     }
   }
-  xm[cq * kRows + r] = mx * sc;                         // scale > 0: the maximum commutes with it
-  __syncthreads();
-  float m_run = -INFINITY;
+  float m_run = mx * sc;                                // scale > 0: the maximum commutes with it
+  if (NQ > 1) {
+    xm[cq * kRows + r] = m_run;
+    __syncthreads();
 #pragma unroll
-  for (int u = 0; u < NQ; ++u) m_run = fmaxf(m_run, xm[u * kRows + r]);
+    for (int u = 0; u < NQ; ++u) m_run = fmaxf(m_run, xm[u * kRows + r]);
+  }
   // m_run is finite: at least one parent holds a key.
   PHASE_MARK(4);
 
-  // ---- fp32 weights parked in TMEM; exact denominator of the parent pass.  Empty parents need no
-  // zeroing: the clamp keeps their weight finite and their count and value sum are zero.
+  // ---- fp32 weights; exact denominator of the parent pass.  Empty parents need no zeroing: the clamp
+  // keeps their weight finite and their count and value sum are zero.
+  float zfull = 0.f;
   {
     const float negm = -m_run;
-    float zloc = 0.f;
-    for (int c0 = 0; c0 < my_cols; c0 += 16) {
-      float s[16];
-      tmem_ld16(t_s + c0, s);
-      const float4* n4 = reinterpret_cast<const float4*>(cnt + colbase + c0);
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const float4 n = n4[u];
-        s[4 * u] = ex2(fminf(fmaf(s[4 * u], sc, negm), 0.f));
-        s[4 * u + 1] = ex2(fminf(fmaf(s[4 * u + 1], sc, negm), 0.f));
-        s[4 * u + 2] = ex2(fminf(fmaf(s[4 * u + 2], sc, negm), 0.f));
-        s[4 * u + 3] = ex2(fminf(fmaf(s[4 * u + 3], sc, negm), 0.f));
-        zloc = fmaf(s[4 * u], n.x, zloc);
-        zloc = fmaf(s[4 * u + 1], n.y, zloc);
-        zloc = fmaf(s[4 * u + 2], n.z, zloc);
-        zloc = fmaf(s[4 * u + 3], n.w, zloc);
+    for (int c0 = 0; c0 < QW; c0 += 16) {
+      if (c0 < my_cols) {
+        const float4* n4 = reinterpret_cast<const float4*>(cnt + colbase + c0);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float4 n = n4[u];
+          a[c0 + 4 * u] = ex2(fminf(fmaf(a[c0 + 4 * u], sc, negm), 0.f));
+          a[c0 + 4 * u + 1] = ex2(fminf(fmaf(a[c0 + 4 * u + 1], sc, negm), 0.f));
+          a[c0 + 4 * u + 2] = ex2(fminf(fmaf(a[c0 + 4 * u + 2], sc, negm), 0.f));
+          a[c0 + 4 * u + 3] = ex2(fminf(fmaf(a[c0 + 4 * u + 3], sc, negm), 0.f));
+          zfull = fmaf(a[c0 + 4 * u], n.x, zfull);
+          zfull = fmaf(a[c0 + 4 * u + 1], n.y, zfull);
+          zfull = fmaf(a[c0 + 4 * u + 2], n.z, zfull);
+          zfull = fmaf(a[c0 + 4 * u + 3], n.w, zfull);
+        }
       }
-      tmem_st16(t_s + c0, s);
     }
-    tmem_st_wait();
-    xz[cq * kRows + r] = zloc;
+    if (NQ > 1) {
+      xz[cq * kRows + r] = zfull;
+      __syncthreads();
+      zfull = 0.f;
+#pragma unroll
+      for (int u = 0; u < NQ; ++u) zfull += xz[u * kRows + r];
+    }
   }
-  __syncthreads();
   PHASE_MARK(5);
   {
-    float zfull = 0.f;
-#pragma unroll
-    for (int u = 0; u < NQ; ++u) zfull += xz[u * kRows + r];
     const float inv = (r < rows_valid) ? 1.f / zfull : 0.f;
     // ---- importance: column sums of A_ij / z_i over the 128 rows (32 per warp, then 4 warps)
-    if ((QW & 31) == 0) {
-      for (int c0 = 0; c0 < my_cols; c0 += 32) {
-        float v[32];
-        float a[16];
-        tmem_ld16(t_s + c0, a);
+    if constexpr ((QW & 31) == 0) {
 #pragma unroll
-        for (int e = 0; e < 16; ++e) v[e] = a[e] * inv;
-        tmem_ld16(t_s + c0 + 16, a);
+      for (int c0 = 0; c0 < QW; c0 += 32) {
+        if (c0 < my_cols) {
+          float v[32];
 #pragma unroll
-        for (int e = 0; e < 16; ++e) v[16 + e] = a[e] * inv;
-        const float colsum = transpose_reduce<32>(v, lane);
-        wpart[q * CT + colbase + c0 + lane] = colsum;
+          for (int e = 0; e < 32; ++e) v[e] = a[c0 + e] * inv;
+          const float colsum = transpose_reduce<32>(v, lane);
+          wpart[q * CT + colbase + c0 + lane] = colsum;
+        }
       }
     } else {
-      for (int c0 = 0; c0 < my_cols; c0 += 16) {
-        float v[16];
-        tmem_ld16(t_s + c0, v);
 #pragma unroll
-        for (int e = 0; e < 16; ++e) v[e] *= inv;
-        const float colsum = transpose_reduce<16>(v, lane);
-        if ((lane & 1) == 0) wpart[q * CT + colbase + c0 + (lane >> 1)] = colsum;
+      for (int c0 = 0; c0 < QW; c0 += 16) {
+        if (c0 < my_cols) {
+          float v[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) v[e] = a[c0 + e] * inv;
+          const float colsum = transpose_reduce<16>(v, lane);
+          if ((lane & 1) == 0) wpart[q * CT + colbase + c0 + (lane >> 1)] = colsum;
+        }
       }
     }
   }
@@ -426,19 +440,21 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // ---- masked bf16 weights into shared memory (over the dead codebook) + their denominator
   {
     float zloc = 0.f;
-    for (int c0 = 0; c0 < my_cols; c0 += 16) {
-      float a[16];
-      tmem_ld16(t_s + c0, a);
-      const float4* k4 = reinterpret_cast<const float4*>(keep + colbase + c0);
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const float4 kk = k4[u];
-        a[4 * u] *= kk.x;
-        a[4 * u + 1] *= kk.y;
-        a[4 * u + 2] *= kk.z;
-        a[4 * u + 3] *= kk.w;
+    for (int c0 = 0; c0 < QW; c0 += 16) {
+      if (c0 < my_cols) {
+        float am[16];
+        const float4* k4 = reinterpret_cast<const float4*>(keep + colbase + c0);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float4 kk = k4[u];
+          am[4 * u] = a[c0 + 4 * u] * kk.x;
+          am[4 * u + 1] = a[c0 + 4 * u + 1] * kk.y;
+          am[4 * u + 2] = a[c0 + 4 * u + 2] * kk.z;
+          am[4 * u + 3] = a[c0 + 4 * u + 3] * kk.w;
+        }
+        zloc += store_weights16(CA, r, colbase + c0, cnt + colbase + c0, am);
       }
-      zloc += store_weights16(CA, r, colbase + c0, cnt + colbase + c0, a);
     }
     xz2[cq * kRows + r] = zloc;
   }
