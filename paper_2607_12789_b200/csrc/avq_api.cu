@@ -148,9 +148,10 @@ Regions carve(void* workspace, const Layout& L) {
 }
 avq_status attend_stage(const avq_problem& p, const Regions& r, const void* Q, const void* Cp, const void* Cc,
                         int32_t P, int32_t block_q, void* Y, int32_t* topp_out, float* importance_out,
-                        cudaStream_t st) {
+                        bool chained, cudaStream_t st) {
   if (use_tensor_path(p))
-    return tc_attend(p, Q, Cp, Cc, r.np_, r.nc, r.VpT, r.VcT, P, Y, topp_out, importance_out, r.status_word, st);
+    return tc_attend(p, Q, Cp, Cc, r.np_, r.nc, r.VpT, r.VcT, P, Y, topp_out, importance_out, r.status_word,
+                     chained, st);
   return simt_attend(p, Q, Cp, Cc, r.Vp, r.np_, r.Vc, r.nc, P, block_q, Y, topp_out, importance_out, st);
 }
 avq_status check_workspace(const avq_problem* prob, int32_t P, int32_t block_q, void* workspace,
@@ -192,7 +193,7 @@ avq_status avq_forward(const avq_problem* prob, const void* Q, const void* K, co
     s = simt_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, st);
   }
   if (s != AVQ_OK) return s;
-  return attend_stage(p, r, Q, Cp, Cc, P, block_q, Y, topp_out, importance_out, st);
+  return attend_stage(p, r, Q, Cp, Cc, P, block_q, Y, topp_out, importance_out, true, st);
 }
 
 avq_status avq_attend(const avq_problem* prob, const void* Q, const void* Cp, const void* Cc, int32_t P,
@@ -207,7 +208,7 @@ avq_status avq_attend(const avq_problem* prob, const void* Q, const void* Cp, co
   Layout L;
   s = check_workspace(prob, P, block_q, workspace, workspace_bytes, &L);
   if (s != AVQ_OK) return s;
-  return attend_stage(*prob, carve(workspace, L), Q, Cp, Cc, P, block_q, Y, topp_out, importance_out,
+  return attend_stage(*prob, carve(workspace, L), Q, Cp, Cc, P, block_q, Y, topp_out, importance_out, false,
                       static_cast<cudaStream_t>(stream));
 }
 

@@ -56,7 +56,7 @@ avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* pare
 avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc,
                      const float* np_, const float* nc, const void* VpT, const void* VcT, int32_t P,
                      void* Y, int32_t* topp_out, float* importance_out, int32_t* status_word,
-                     cudaStream_t st);
+                     bool chained, cudaStream_t st);   // chained: launched right behind tc_aggregate
 
 inline avq_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? AVQ_OK : AVQ_ERR_CUDA; }
 

@@ -26,6 +26,8 @@ __global__ void __launch_bounds__(kScatterThreads)
 leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restrict__ pidx,
                     const int32_t* __restrict__ cidx, float* __restrict__ Vc, float* __restrict__ nc,
                     int Nk, int M, int C) {
+  tc::pdl_launch_dependents();
+  tc::pdl_wait();                                    // the indices come from the kernel before
   const int bh = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int j0 = blockIdx.x * kKeysPerCta + warp * kKeysPerWarp;
@@ -71,6 +73,8 @@ __global__ void __launch_bounds__(D)
 finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, float* __restrict__ Vp,
                 float* __restrict__ np_, __nv_bfloat16* __restrict__ VpT, __nv_bfloat16* __restrict__ VcT,
                 int M) {
+  tc::pdl_launch_dependents();
+  tc::pdl_wait();                                    // the leaf sums come from the kernel before
   const int bh = blockIdx.y, m0 = blockIdx.x * 8, k = threadIdx.x;
   __align__(16) __nv_bfloat16 pk[8];
 #pragma unroll
@@ -119,13 +123,15 @@ avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const i
     if (cudaMemsetAsync(nc, 0, sizeof(float) * (size_t)BH * p.M * C, st) != cudaSuccess) return AVQ_ERR_CUDA;
   }
   dim3 g1((p.Nk + kKeysPerCta - 1) / kKeysPerCta, BH);
-  leaf_scatter_kernel<D><<<g1, kScatterThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(V), pidx, cidx, Vc,
-                                                         nc, p.Nk, p.M, C);
-  if (cudaGetLastError() != cudaSuccess) return AVQ_ERR_CUDA;
+  // `pre_zeroed` marks the chained call from avq_forward: the kernel before in the stream is the assign
+  // kernel, so the scatter may be launched as its programmatic dependent.
+  if (tc::launch_pdl(leaf_scatter_kernel<D>, g1, dim3(kScatterThreads), 0, st, pre_zeroed,
+                     static_cast<const __nv_bfloat16*>(V), pidx, cidx, Vc, nc, p.Nk, p.M, C) != cudaSuccess)
+    return AVQ_ERR_CUDA;
   dim3 g2(p.M / 8, BH);
-  finalize_kernel<D, C><<<g2, D, 0, st>>>(Vc, nc, Vp, np_, static_cast<__nv_bfloat16*>(VpT),
-                                          static_cast<__nv_bfloat16*>(VcT), p.M);
-  return cuda_ok(cudaGetLastError());
+  return cuda_ok(tc::launch_pdl(finalize_kernel<D, C>, g2, dim3(D), 0, st, true, static_cast<const float*>(Vc),
+                                static_cast<const float*>(nc), Vp, np_, static_cast<__nv_bfloat16*>(VpT),
+                                static_cast<__nv_bfloat16*>(VcT), p.M));
 }
 
 }  // namespace

@@ -116,6 +116,7 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   const int MH = M >> 1;                             // columns per half (multiple of 16: M % 32 == 0)
 
   APHASE(0);
+  pdl_launch_dependents();   // the next kernel of the call may begin its set-up
   if (tid == 0) {
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmCp);

@@ -162,13 +162,12 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   uint64_t* bar_s = &bars[2];
   uint64_t* bar_pv = &bars[3];
 
-  // A wait that expired in an earlier CTA of this launch: do not start more work.
-  // The flag is read here and acted on after the set-up barrier below, so that it costs no extra round trip.
   __shared__ int early_exit;
-  if (tid == 0) early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
   PHASE_MARK(0);
 
-  // ---- barriers, then the loads first: Q tile + parent codebook, and the parents' value sums
+  // ---- Part 1 touches only the caller's Q and Cp, so it may run while the kernel that produces the
+  // aggregates is still finishing (programmatic dependent launch): barriers, TMEM, the Q / Cp loads and
+  // S = Q . Cp^T.
   if (tid == 0) {
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmCp);
@@ -185,32 +184,15 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       tma_load_3d(Qs + s * kRows * 128, &tmQ, s * 64, i0, bh, bar_ld0);
       tma_load_2d(CA + s * M * 128, &tmCp, s * 64, h * M, bar_ld0);
     }
-    const int subM = (M + 63) >> 6;
-    mbar_expect_tx(bar_ld1, (uint32_t)(subM * D * 128));
-    for (int s = 0; s < subM; ++s) tma_load_2d(Vs + s * D * 128, &tmVpT, s * 64, bh * D, bar_ld1);
   }
   if (warp == 0) {
     tmem_alloc(tmem_slot, p.tmem_cols);
     tmem_relinquish();
   }
-  for (int j = tid; j < CT; j += kThreads) {
-    const float n = j < M ? p.np_[(size_t)bh * M + j] : 0.f;
-    cnt[j] = n;
-    bias[j] = n > 0.f ? 0.f : -INFINITY;
-    keep[j] = 1.f;
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  if (early_exit) {
-    // let the loads already in flight land in this CTA's shared memory, then leave cleanly
-    mbar_wait(bar_ld0, 0, abort_flag, nullptr, 0);
-    mbar_wait(bar_ld1, 0, abort_flag, nullptr, 0);
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
-    return;
-  }
   const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
   const uint32_t t_s = t_row + (uint32_t)colbase;
   const uint32_t t_sc = t_row + (uint32_t)(cq * QWC);
@@ -218,8 +200,6 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const uint32_t idesc_o = umma_idesc_bf16(kRows, D);
   const float sc = p.scale_log2e;
   PHASE_MARK(1);
-
-  // ---- S = Q . Cp^T
   if (tid == 0) {
     if (mbar_wait(bar_ld0, 0, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND)) {
       tc_fence_after();
@@ -229,8 +209,34 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       for (int k = 0; k < D / 16; ++k)
         umma_bf16(tmem_base, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
                   umma_desc_sw128(ca + (k / 4) * M * 128 + (k % 4) * 32), idesc, k > 0);
-      umma_commit(bar_s);
     }
+    umma_commit(bar_s);
+  }
+
+  // ---- Part 2 reads what the earlier kernels of this call wrote: status word, counts, value sums.
+  pdl_wait();
+  if (tid == 0) {
+    // a wait that expired in an earlier CTA or kernel of this call: do not start more work
+    early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
+    const int subM = (M + 63) >> 6;
+    mbar_expect_tx(bar_ld1, (uint32_t)(subM * D * 128));
+    for (int s = 0; s < subM; ++s) tma_load_2d(Vs + s * D * 128, &tmVpT, s * 64, bh * D, bar_ld1);
+  }
+  for (int j = tid; j < CT; j += kThreads) {
+    const float n = j < M ? p.np_[(size_t)bh * M + j] : 0.f;
+    cnt[j] = n;
+    bias[j] = n > 0.f ? 0.f : -INFINITY;
+    keep[j] = 1.f;
+  }
+  __syncthreads();
+  if (early_exit) {
+    // let the MMA and the load already in flight finish, then leave cleanly
+    mbar_wait(bar_s, 0, abort_flag, nullptr, 0);
+    mbar_wait(bar_ld1, 0, abort_flag, nullptr, 0);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+    return;
   }
   uint32_t ph_s = 0, ph_pv = 0;
   const int PC = P * C;
@@ -654,7 +660,8 @@ size_t attend_smem(int D, int CT, int CHW, int NQ) {
 
 template <int D, int NQ, int CT>
 avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUtensorMap& tmVpT,
-                     const CUtensorMap& tmY, const AttendParams& a, unsigned BH, size_t smem, cudaStream_t st) {
+                     const CUtensorMap& tmY, const AttendParams& a, unsigned BH, size_t smem, bool chained,
+                     cudaStream_t st) {
   auto kern = tc_attend_kernel<D, NQ, CT>;
   // The limit is set once per device and instantiation (setting it again is harmless if two threads race).
   static size_t configured[64] = {};
@@ -666,14 +673,16 @@ avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUte
     if (dev >= 0 && dev < 64) configured[dev] = smem;
   }
   dim3 grid(a.nblk, BH);
-  kern<<<grid, 128 * NQ, smem, st>>>(tmQ, tmCp, tmVpT, tmY, a);
-  return cuda_ok(cudaGetLastError());
+  // Inside avq_forward (`chained`) the kernel before it in the stream is the aggregate's finalize kernel
+  // and Q was complete before the call, so the attention kernel may start as its programmatic dependent.
+  // A stand-alone avq_attend is launched plainly: the work before it in the stream may be producing Q.
+  return cuda_ok(launch_pdl(kern, grid, dim3(128 * NQ), smem, st, chained, tmQ, tmCp, tmVpT, tmY, a));
 }
 
 template <int D>
 avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const void* Cc, const float* np_,
                   const float* nc, const void* VpT, const void* VcT, int32_t P, void* Y, int32_t* topp_out,
-                  float* importance_out, int32_t* status_word, cudaStream_t st) {
+                  float* importance_out, int32_t* status_word, bool chained, cudaStream_t st) {
   const uint64_t BH = (uint64_t)p.B * p.H;
   CUtensorMap tmQ, tmCp, tmVpT, tmY;
   {
@@ -720,13 +729,13 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
   // four small CTAs of 128 threads, two of 256, or one of 512.
   const unsigned bh = (unsigned)BH;
   if (D == 64) {
-    if (CT == 64) return launch_nq<D, 1, 64>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
-    if (CT == 128) return launch_nq<D, 2, 128>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
-    return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
+    if (CT == 64) return launch_nq<D, 1, 64>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
+    if (CT == 128) return launch_nq<D, 2, 128>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
+    return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
   }
-  if (CT == 64) return launch_nq<D, 2, 64>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
-  if (CT == 128) return launch_nq<D, 4, 128>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
-  return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, st);
+  if (CT == 64) return launch_nq<D, 2, 64>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
+  if (CT == 128) return launch_nq<D, 4, 128>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
+  return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
 }
 
 }  // namespace
@@ -739,9 +748,9 @@ extern "C" __attribute__((visibility("default"))) int avq_debug_phase_clocks(lon
 
 avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc, const float* np_,
                      const float* nc, const void* VpT, const void* VcT, int32_t P, void* Y, int32_t* topp_out,
-                     float* importance_out, int32_t* status_word, cudaStream_t st) {
-  return p.d == 64 ? launch<64>(p, Q, Cp, Cc, np_, nc, VpT, VcT, P, Y, topp_out, importance_out, status_word, st)
-                   : launch<128>(p, Q, Cp, Cc, np_, nc, VpT, VcT, P, Y, topp_out, importance_out, status_word, st);
+                     float* importance_out, int32_t* status_word, bool chained, cudaStream_t st) {
+  return p.d == 64 ? launch<64>(p, Q, Cp, Cc, np_, nc, VpT, VcT, P, Y, topp_out, importance_out, status_word, chained, st)
+                   : launch<128>(p, Q, Cp, Cc, np_, nc, VpT, VcT, P, Y, topp_out, importance_out, status_word, chained, st);
 }
 
 }  // namespace avq
