@@ -21,8 +21,8 @@
  * Conventions
  *   - Every pointer is a DEVICE pointer unless the argument is documented as host.
  *     The caller owns every buffer.  The library allocates no device memory and keeps
- *     no mutable global state; calls on different streams with different workspaces
- *     may overlap.
+ *     no state that can change a result (it caches encoded TMA descriptors and one-time
+ *     kernel attributes); calls on different streams with different workspaces may overlap.
  *   - All tensors are dense, row-major, last index fastest:
  *       Q  [B, H, Nq, d]     K, V [B, H, Nk, d]     Y [B, H, Nq, d]
  *       Cp [H, M, d]         parent codebook, one per head, shared over the batch
