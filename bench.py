@@ -129,7 +129,7 @@ class ClockSampler:
                     window="warm-up, timed steps and 1 s more of the same step")
 
 
-def run_gpu(wl, steps, warmup, rank, world, flags=0, extras=True, min_warm_s=0.3):
+def run_gpu(wl, steps, warmup, rank, world, flags=0, extras=True, min_warm_s=0.3, spin=True):
     import torch
     from paper_2607_12789_b200 import binding, synth
     dev = torch.device("cuda", torch.cuda.current_device())
@@ -158,7 +158,7 @@ def run_gpu(wl, steps, warmup, rank, world, flags=0, extras=True, min_warm_s=0.3
         # end-to-end loop (whose host work is part of what is measured) runs without it.
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
-        if head_start:
+        if head_start and spin:
             torch.cuda._sleep(int(2.0e6 * min(n, 64) / 10))
         e0.record()
         for i in range(n):
@@ -342,7 +342,7 @@ def main():
                                           forward_roofline_frac=fr2["frac"])), flush=True)
         return
     if args.profile:
-        res = run_gpu(wl, args.steps, warm, rank, world, flags=flags, extras=False, min_warm_s=0.0)
+        res = run_gpu(wl, args.steps, warm, rank, world, flags=flags, extras=False, min_warm_s=0.0, spin=False)
         if rank == 0:
             print(json.dumps(dict(metric=METRIC, profile_only=True, ms_per_step=res["ms"], config=config)))
         return
