@@ -90,6 +90,26 @@ def roof(entry, pk, ms, dtype):
     return dict(bound="tensor", achieved=ach, peak=tflops_peak, unit="TFLOP/s", frac=ach / tflops_peak)
 
 
+def shard_workload(wl, rank: int):
+    """Weak scaling: every rank runs its own batch of the same shape (its own seed), no data exchange."""
+    return wl.with_(seed=wl.seed + 7919 * rank)
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Step time of the job = the slowest rank's (one MAX all-reduce of a scalar; nothing else is exchanged)."""
+    if world <= 1:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(wl, world: int, ms: float) -> float:
+    """Query tokens per second of the whole job (all ranks)."""
+    return wl.B * wl.N * world / (ms * 1e-3)
+
+
 class ClockSampler:
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -134,7 +154,7 @@ def run_gpu(wl, steps, warmup, rank, world, flags=0, extras=True, min_warm_s=0.3
     from paper_2607_12789_b200 import binding, synth
     dev = torch.device("cuda", torch.cuda.current_device())
     td = torch.float32 if wl.dtype == "f32" else torch.bfloat16
-    x = synth.generate(wl.with_(seed=wl.seed + 7919 * rank))
+    x = synth.generate(shard_workload(wl, rank))
     host = {k: torch.from_numpy(v).to(td) for k, v in x.items()}
     l2 = torch.cuda.get_device_properties(dev).L2_cache_size
     foot = sum(host[k].numel() * host[k].element_size() for k in "QKV") + host["Q"].numel() * host["Q"].element_size()
@@ -182,10 +202,7 @@ def run_gpu(wl, steps, warmup, rank, world, flags=0, extras=True, min_warm_s=0.3
     barrier()
     ms = timed(step, steps)
     barrier()
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, dev)
     f.check()
     out = dict(ms=ms, copies=copies, footprint_mb=foot * copies / 1e6, l2_mb=l2 / 1e6)
     if not extras:
@@ -239,10 +256,7 @@ def run_gpu(wl, steps, warmup, rank, world, flags=0, extras=True, min_warm_s=0.3
     barrier()
     e2e_ms = timed(e2e_fn, steps, head_start=False)
     barrier()
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, dev)
     f.check()
     es = hq.element_size()
     out["e2e"] = dict(ms=e2e_ms, h2d=3 * hq.numel() * es, d2h=hq.numel() * es,
@@ -349,7 +363,7 @@ def main():
     res = run_gpu(wl, args.steps, warm, rank, world, flags=flags)
     ms = res["ms"]
     tokens = wl.B * wl.N * world
-    value = tokens / (ms * 1e-3)
+    value = job_value(wl, world, ms)
     dom = max(res["stages_ms"], key=res["stages_ms"].get)
     rl = roof(stage_model[dom], pk, res["stages_ms"][dom], wl.dtype)
     rl.update(kernel=dom, traffic=None, peak_source=pk["source"],
