@@ -85,6 +85,13 @@ __device__ __forceinline__ float transpose_reduce(float (&v)[V], int lane) {
   return v[0];
 }
 
+// The NQ warps that share a quarter of the rows (warp % 4 == q) exchange per-row values through shared
+// memory; they synchronise among themselves on named barrier q + 1 instead of stalling the whole CTA.
+template <int NQ>
+__device__ __forceinline__ void row_sync(int q) {
+  asm volatile("bar.sync %0, %1;" ::"r"(q + 1), "r"(32 * NQ) : "memory");
+}
+
 // Rounds 16 fp32 weights to bf16, stores them at (row r, columns col0..col0+15) of the K-major
 // swizzled A tile, and returns sum(rounded weight * count).
 __device__ __forceinline__ float store_weights16(unsigned char* A, int r, int col0, const float* cnt16,
@@ -274,7 +281,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   float m_run = mx * sc;                                // scale > 0: the maximum commutes with it
   if (NQ > 1) {
     xm[cq * kRows + r] = m_run;
-    __syncthreads();
+    row_sync<NQ>(q);
 #pragma unroll
     for (int u = 0; u < NQ; ++u) m_run = fmaxf(m_run, xm[u * kRows + r]);
   }
@@ -306,7 +313,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
     if (NQ > 1) {
       xz[cq * kRows + r] = zfull;
-      __syncthreads();
+      row_sync<NQ>(q);
       zfull = 0.f;
 #pragma unroll
       for (int u = 0; u < NQ; ++u) zfull += xz[u * kRows + r];
@@ -543,11 +550,13 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         mxc = fmaxf(mxc, fmaxf(s[4 * u + 2] + b.z, s[4 * u + 3] + b.w));
       }
     }
-    xm[cq * kRows + r] = mxc * sc;
-    __syncthreads();
-    float m_new = m_run;
+    float m_new = fmaxf(m_run, mxc * sc);
+    if (NQ > 1) {
+      xm[cq * kRows + r] = mxc * sc;
+      row_sync<NQ>(q);
 #pragma unroll
-    for (int u = 0; u < NQ; ++u) m_new = fmaxf(m_new, xm[u * kRows + r]);
+      for (int u = 0; u < NQ; ++u) m_new = fmaxf(m_new, xm[u * kRows + r]);
+    }
     const float negm = -m_new;
     if (e0 == 0) PHASE_MARK(14);
     // ---- rescale what has been accumulated if this row's maximum moved
