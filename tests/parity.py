@@ -119,12 +119,23 @@ def sampled_parity(wl: synth.Workload, heads, blocks_per_head: int = 8, flags: i
         rep["child_flips_excused"] += r["child_flips_excused"]
         if r["parent_flips_excused"] == 0 and r["child_flips_excused"] == 0:
             compare_aggregates(gh, ref)
+        # importance and selection of EVERY block of the head (cheap for the oracle: no O(N^2) part)
+        n_all = 0
+        for t in range(nblk):
+            Qb = x["Q"][b, h][t * wl.block_q:(t + 1) * wl.block_q]
+            w_or, _, _, _ = orc.importance_block(Qb, x["Cp"][h], ref["np"], wl.scale)
+            sel_or, margin = orc.top_p(w_or, wl.P)
+            if not np.array_equal(gh["selected"][t], sel_or):
+                assert margin < NEAR_TIE, f"head {(b, h)} block {t}: wrong top-P set at margin {margin:.2e}"
+                rep["topp_flips_excused"] += 1
+            assert np.allclose(gh["importance"][t], w_or, rtol=2e-3, atol=2e-4)
+            n_all += 1
+        rep["blocks_selection_checked"] = rep.get("blocks_selection_checked", 0) + n_all
         sub = dict(selected=gh["selected"][blocks], importance=gh["importance"][blocks])
         same, excused = compare_selection(sub, dict(selected=ref["selected"][blocks],
                                                     importance=ref["importance"][blocks],
                                                     topp_margin=ref["topp_margin"][blocks]))
-        rep["topp_flips_excused"] += excused
-        for t, ok in zip(blocks, same):
+        for t, ok in zip(blocks, same):     # `excused` is already counted by the all-block loop above
             if not ok:
                 continue
             rows = slice(t * wl.block_q, min(wl.N, (t + 1) * wl.block_q))
