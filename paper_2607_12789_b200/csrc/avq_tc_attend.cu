@@ -320,7 +320,10 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
   }
   PHASE_MARK(5);
-  {
+  // The importances are needed only to choose which parents to refine: with P = 0 (nothing refined) or
+  // P >= M (everything refined) the choice is fixed and the pass is skipped unless the caller wants them.
+  const bool need_w = (P > 0 && P < M) || p.importance_out != nullptr;
+  if (need_w) {
     const float inv = (r < rows_valid) ? 1.f / zfull : 0.f;
     // ---- importance: column sums of A_ij / z_i over the 128 rows (32 per warp, then 4 warps)
     if constexpr ((QW & 31) == 0) {
@@ -347,14 +350,16 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
     }
   }
-  __syncthreads();
-  PHASE_MARK(6);
-  if (tid < M) {
-    const float wj = cnt[tid] * ((wpart[tid] + wpart[CT + tid]) + (wpart[2 * CT + tid] + wpart[3 * CT + tid]));
-    w[tid] = wj;
-    if (p.importance_out) p.importance_out[((size_t)bh * p.nblk + blk) * M + tid] = wj;
+  if (need_w) {
+    __syncthreads();
+    PHASE_MARK(6);
+    if (tid < M) {
+      const float wj = cnt[tid] * ((wpart[tid] + wpart[CT + tid]) + (wpart[2 * CT + tid] + wpart[3 * CT + tid]));
+      w[tid] = wj;
+      if (p.importance_out) p.importance_out[((size_t)bh * p.nblk + blk) * M + tid] = wj;
+    }
+    __syncthreads();
   }
-  __syncthreads();
   PHASE_MARK(7);
 
   // ---- top-P by rank.  Non-negative floats order like their bit patterns, so the comparisons run on
