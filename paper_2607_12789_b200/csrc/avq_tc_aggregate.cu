@@ -66,6 +66,127 @@ leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restri
   if (leaf_l >= 0) atomicAdd(nc + (size_t)bh * M * C + leaf_l, 1.0f);
 }
 
+// Long sequences over few codewords put hundreds of keys on every leaf, and the reductions above then
+// queue on the same addresses.  This variant gives one CTA a contiguous chunk of a head's keys, orders
+// the chunk by leaf with a counting sort in shared memory (integer atomics only) and lets every warp walk
+// an equal share of the ordered list, summing in registers: a leaf costs one global reduction per CTA
+// (one more where a leaf straddles two warps' shares) instead of one per key.
+constexpr int kSortThreads = 512;
+constexpr int kSortKeysPerThread = 16;
+constexpr int kSortMaxKeys = kSortThreads * kSortKeysPerThread;   // keys per CTA (16-bit key field of the order list)
+constexpr int kSortMaxLeaves = 2048;                              // M * C <= 256 * 8
+constexpr int kSortRatio = 2;                                     // chunked variant from this many keys per leaf
+
+template <int D>
+__global__ void __launch_bounds__(kSortThreads, 2)
+leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restrict__ pidx,
+                   const int32_t* __restrict__ cidx, float* __restrict__ Vc, float* __restrict__ nc,
+                   int Nk, int L, int C, int chunk) {
+  extern __shared__ __align__(16) unsigned char sort_smem[];
+  int* hist = reinterpret_cast<int*>(sort_smem);        // [L] keys per leaf
+  int* offs = hist + L;                                 // [L] first slot of each leaf in `order`
+  int* wsum = offs + L;                                 // [16] per-warp totals of the scan
+  uint32_t* order = reinterpret_cast<uint32_t*>(wsum + 16);   // [chunk] leaf << 16 | key (relative to the chunk)
+  tc::pdl_launch_dependents();
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bh = blockIdx.y;
+  const int j0 = blockIdx.x * chunk;
+  const int n = min(chunk, Nk - j0);
+  for (int l = tid; l < L; l += kSortThreads) hist[l] = 0;
+  __syncthreads();
+  tc::pdl_wait();                                      // the indices come from the kernel before
+  if (n <= 0) return;
+  const size_t kb = (size_t)bh * Nk + j0;
+
+  // ---- leaf of every key and its rank among the chunk's keys of that leaf
+  uint32_t lr[kSortKeysPerThread];                     // leaf << 16 | rank
+#pragma unroll
+  for (int t = 0; t < kSortKeysPerThread; ++t) {
+    const int j = tid + t * kSortThreads;
+    lr[t] = 0xFFFFFFFFu;
+    if (j < n) {
+      const int leaf = __ldg(pidx + kb + j) * C + __ldg(cidx + kb + j);
+      lr[t] = ((uint32_t)leaf << 16) | (uint32_t)atomicAdd(&hist[leaf], 1);
+    }
+  }
+  __syncthreads();
+
+  // ---- exclusive scan of the histogram: thread t owns entries [t * E, (t + 1) * E); key counts go out
+  {
+    const int E = (L + kSortThreads - 1) / kSortThreads;   // <= 4
+    int c[4] = {0, 0, 0, 0}, tot = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (e < E && tid * E + e < L) {
+        c[e] = hist[tid * E + e];
+        tot += c[e];
+        if (c[e] > 0) atomicAdd(nc + (size_t)bh * L + tid * E + e, (float)c[e]);
+      }
+    int inc = tot;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += up;
+    }
+    if (lane == 31) wsum[warp] = inc;
+    __syncthreads();
+    int base = inc - tot;
+    for (int u = 0; u < warp; ++u) base += wsum[u];
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (e < E && tid * E + e < L) { offs[tid * E + e] = base; base += c[e]; }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int t = 0; t < kSortKeysPerThread; ++t)
+    if (lr[t] != 0xFFFFFFFFu)
+      order[offs[lr[t] >> 16] + (int)(lr[t] & 0xFFFFu)] = (lr[t] & 0xFFFF0000u) | (uint32_t)(tid + t * kSortThreads);
+  __syncthreads();
+
+  // ---- every warp walks an equal share of the ordered list, 16 rows in flight (lane = 2 or 4 consecutive
+  // head dimensions), and flushes its register sum whenever the leaf changes
+  using Word = typename std::conditional<D == 64, uint32_t, uint2>::type;
+  const Word* Vw = reinterpret_cast<const Word*>(V + kb * D) + lane;   // row j at Vw + j * 32
+  constexpr int kWarps = kSortThreads / 32, kBatch = 16;
+  const int share = (n + kWarps - 1) / kWarps;
+  const int s0 = warp * share, s1 = min(n, s0 + share);
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  int cur = -1;
+  auto flush = [&]() {
+    if (cur < 0) return;
+    float* dst = Vc + ((size_t)bh * L + cur) * D;
+    if constexpr (D == 64) atomicAdd(reinterpret_cast<float2*>(dst) + lane, make_float2(acc[0], acc[1]));
+    else atomicAdd(reinterpret_cast<float4*>(dst) + lane, make_float4(acc[0], acc[1], acc[2], acc[3]));
+    acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+  };
+  for (int i = s0; i < s1; i += kBatch) {
+    uint32_t e[kBatch];
+    Word w[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      e[u] = order[min(i + u, s1 - 1)];
+      w[u] = __ldg(Vw + (size_t)(e[u] & 0xFFFFu) * 32);
+    }
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      if (i + u < s1) {                                // warp-uniform
+        const int leaf = (int)(e[u] >> 16);
+        if (leaf != cur) { flush(); cur = leaf; }
+        if constexpr (D == 64) {
+          acc[0] += __uint_as_float(w[u] << 16);
+          acc[1] += __uint_as_float(w[u] & 0xFFFF0000u);
+        } else {
+          acc[0] += __uint_as_float(w[u].x << 16);
+          acc[1] += __uint_as_float(w[u].x & 0xFFFF0000u);
+          acc[2] += __uint_as_float(w[u].y << 16);
+          acc[3] += __uint_as_float(w[u].y & 0xFFFF0000u);
+        }
+      }
+    }
+  }
+  flush();
+}
+
 // One CTA: 8 consecutive parents of one (batch, head); thread k owns head-dimension index k.
 // All loads of four parents are issued before their first use.
 template <int D, int C>
@@ -122,12 +243,49 @@ avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const i
     if (cudaMemsetAsync(Vc, 0, sizeof(float) * (size_t)BH * p.M * C * D, st) != cudaSuccess) return AVQ_ERR_CUDA;
     if (cudaMemsetAsync(nc, 0, sizeof(float) * (size_t)BH * p.M * C, st) != cudaSuccess) return AVQ_ERR_CUDA;
   }
-  dim3 g1((p.Nk + kKeysPerCta - 1) / kKeysPerCta, BH);
   // `pre_zeroed` marks the chained call from avq_forward: the kernel before in the stream is the assign
   // kernel, so the scatter may be launched as its programmatic dependent.
-  if (tc::launch_pdl(leaf_scatter_kernel<D>, g1, dim3(kScatterThreads), 0, st, pre_zeroed,
-                     static_cast<const __nv_bfloat16*>(V), pidx, cidx, Vc, nc, p.Nk, p.M, C) != cudaSuccess)
-    return AVQ_ERR_CUDA;
+  // Chunked variant when a CTA's share of a head holds several keys per leaf: about two CTAs per SM.
+  const int L = p.M * C;
+  int sms = 148;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return AVQ_ERR_CUDA;
+    static int cached_sms[64] = {};
+    if (dev >= 0 && dev < 64 && cached_sms[dev] > 0) sms = cached_sms[dev];
+    else {
+      if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return AVQ_ERR_CUDA;
+      if (dev >= 0 && dev < 64) cached_sms[dev] = sms;
+    }
+  }
+  int per_head = 2 * sms / (int)BH;                      // rounded down: the grid must fit in one wave
+  if (per_head < 1) per_head = 1;
+  int chunk = (p.Nk + per_head - 1) / per_head;
+  if (chunk > kSortMaxKeys) chunk = kSortMaxKeys;
+  chunk = (chunk + 31) & ~31;
+  if (L <= kSortMaxLeaves && chunk >= kSortRatio * L) {
+    dim3 g1((p.Nk + chunk - 1) / chunk, BH);
+    const size_t smem = sizeof(int) * (2 * (size_t)L + 16) + sizeof(uint32_t) * (size_t)chunk;
+    // above the default limit only for the largest leaf count and chunk: opt in once per device
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return AVQ_ERR_CUDA;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+      const int max_smem = (int)(sizeof(int) * (2 * kSortMaxLeaves + 16) + sizeof(uint32_t) * kSortMaxKeys);
+      if (cudaFuncSetAttribute(leaf_sorted_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) !=
+          cudaSuccess)
+        return AVQ_ERR_CUDA;
+      if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    if (tc::launch_pdl(leaf_sorted_kernel<D>, g1, dim3(kSortThreads), smem, st, pre_zeroed,
+                       static_cast<const __nv_bfloat16*>(V), pidx, cidx, Vc, nc, p.Nk, L, C, chunk) != cudaSuccess)
+      return AVQ_ERR_CUDA;
+  } else {
+    dim3 g1((p.Nk + kKeysPerCta - 1) / kKeysPerCta, BH);
+    if (tc::launch_pdl(leaf_scatter_kernel<D>, g1, dim3(kScatterThreads), 0, st, pre_zeroed,
+                       static_cast<const __nv_bfloat16*>(V), pidx, cidx, Vc, nc, p.Nk, p.M, C) != cudaSuccess)
+      return AVQ_ERR_CUDA;
+  }
   dim3 g2(p.M / 8, BH);
   return cuda_ok(tc::launch_pdl(finalize_kernel<D, C>, g2, dim3(D), 0, st, true, static_cast<const float*>(Vc),
                                 static_cast<const float*>(nc), Vp, np_, static_cast<__nv_bfloat16*>(VpT),

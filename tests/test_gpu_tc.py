@@ -82,3 +82,28 @@ def test_tensor_core_and_cuda_core_paths_agree_at_full_size():
     rows = same.repeat_interleave(wl.block_q, dim=-1)
     diff = (Yt.float() - Ys.float()).abs()[rows]
     assert diff.max() <= 2e-2
+
+
+@pytest.mark.parametrize("H,N,d,M,C", [(2, 40001, 64, 32, 4), (2, 80003, 128, 32, 8), (16, 16384, 64, 64, 4),
+                                       (1, 1300000, 64, 256, 8)])
+def test_aggregate_long_heads_few_leaves(H, N, d, M, C):
+    """avq_aggregate where every leaf collects many keys (the chunked, leaf-ordered variant), ragged
+    lengths, skewed and empty leaves: counts exact, sums within fp32 accumulation error of the oracle."""
+    from oracle import avq_oracle as orc
+    g = np.random.default_rng(100 + N)
+    V = synth.round_to_bf16(g.standard_normal((1, H, N, d)).astype(np.float32))
+    # skewed leaves: a few popular ones, some never used
+    pm = g.dirichlet(np.full(M, 0.3))
+    pidx = g.choice(M, size=(1, H, N), p=pm).astype(np.int32)
+    cidx = np.minimum(g.geometric(0.5, size=(1, H, N)) - 1, C - 1).astype(np.int32)
+    dev = dict(V=torch.from_numpy(V).cuda().to(torch.bfloat16), p=torch.from_numpy(pidx).cuda(),
+               c=torch.from_numpy(cidx).cuda())
+    Vp, n_p, Vc, n_c = binding.aggregate(dev["V"], dev["p"], dev["c"], M, C)
+    torch.cuda.synchronize()
+    for h in range(H):
+        rVp, rnp, rVc, rnc = orc.aggregate_head(V[0, h], pidx[0, h], cidx[0, h], M, C)
+        assert np.array_equal(n_p[0, h].cpu().numpy(), rnp)
+        assert np.array_equal(n_c[0, h].cpu().numpy(), rnc)
+        scale = 1e-6 * np.sqrt(np.maximum(rnc, 1.0))[..., None] * 50 + 1e-5 * np.abs(rVc)
+        assert (np.abs(Vc[0, h].cpu().numpy() - rVc) <= scale + 1e-4).all()
+        assert np.allclose(Vp[0, h].cpu().numpy(), rVp, rtol=2e-5, atol=2e-3)
