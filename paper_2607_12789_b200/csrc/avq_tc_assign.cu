@@ -10,8 +10,8 @@
 //   child    fp32 direct form sum (k - c)^2 on CUDA cores (2 C d flops per key; a second MMA over all
 //            M C children would cost C times the parent GEMM), float64 recheck for near-ties.  Small
 //            child blocks (C d = 256): the two threads of a key take half of the children each.
-//            Larger ones: a warp fetches a key's contiguous C x d block with coalesced 16-byte loads,
-//            every lane squares its 8 differences and shuffles reduce per child.
+//            Larger ones: four lanes per key, each over a quarter of the head dimension for all C
+//            children (one running sum per child), a transposing butterfly merges the four lanes.
 #include "avq_tc_common.cuh"
 
 namespace avq {
@@ -308,76 +308,84 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       chi[r] = c1;
     }
   } else {
-    // ---- child argmin, one warp per key (16 keys per warp).  A parent's C children are one contiguous
-    // C x d block: NL fully coalesced 16-byte loads per lane fetch it.  Lane l holds 8 elements of child
-    // (t * kChildPerLoad + l / kLanesPerChild) for load t; it squares its 8 differences against the key row,
-    // a butterfly sums them per child, a second butterfly merges (best, index, runner-up) over children.
-    // Loads of the next batch of keys are in flight while the current batch is reduced.
-    {
-      constexpr int kLanesPerChild = D / 8;
-      constexpr int kChildPerLoad = 32 / kLanesPerChild;
-      constexpr int kKB = (NL >= 4) ? 1 : 4 / NL;      // keys per batch: 4 loads per lane in flight per buffer
-      constexpr int kNB = 16 / kKB;                    // batches per warp
-      const int kpos = (lane % kLanesPerChild) * 8;    // first key element this lane compares
-      const int grp = lane / kLanesPerChild;
-      const unsigned char* krow_base = Ks + (kpos >> 6) * (kKeys * 128);
-      const size_t head_base = (size_t)h * M;
-      uint4 buf[2][kKB][NL];
-      auto issue = [&](int bsel, int batch) {
+    // ---- child argmin, four lanes per key: a warp takes 8 keys at a time (two passes over its 16 keys).
+    // Lane s of a key's group covers the 16-byte chunks s, s + 4, ... of the key row and of each of the
+    // parent's C children (the group reads 64 contiguous bytes of a child row per load), keeps one running
+    // sum per child, and a transposing butterfly over the four lanes leaves child s (and s + 4) in lane s.
+    // The loads of the next chunk column are in flight while the current one is squared.
+    constexpr int kC = NL * 256 / D;                   // children per parent (4 or 8)
+    constexpr int kChunks = D / 8;                     // 16-byte chunks per row
+    constexpr int kT = kChunks / 4;                    // chunk columns per lane (2 or 4)
+    constexpr int kSteps = 2 * kT;                     // (pass, chunk column) pairs
+    const int s4 = lane & 3, grp = lane >> 2;
+    const size_t head_base = (size_t)h * M;
+    uint4 buf[2][kC];
+    auto issue = [&](int step, uint4 (&dst)[kC]) {
+      const int key = warp * 16 + (step / kT) * 8 + grp;
+      const uint4* src = reinterpret_cast<const uint4*>(Cc + (head_base + par[key]) * kC * D) + (s4 + 4 * (step % kT));
   #pragma unroll
-        for (int b = 0; b < kKB; ++b) {
-          const int key = warp * 16 + batch * kKB + b;
-          const uint4* src = reinterpret_cast<const uint4*>(Cc + (head_base + par[key]) * C * D) + lane;
+      for (int c = 0; c < kC; ++c) dst[c] = __ldg(src + c * kChunks);
+    };
+    float sum[kC];
+    issue(0, buf[0]);
   #pragma unroll
-          for (int t = 0; t < NL; ++t) buf[bsel][b][t] = __ldg(src + t * 32);
+    for (int step = 0; step < kSteps; ++step) {
+      const int pass = step / kT, t = step % kT;
+      const int key = warp * 16 + pass * 8 + grp;
+      if (step + 1 < kSteps) issue(step + 1, buf[(step + 1) & 1]);
+      if (t == 0) {
+  #pragma unroll
+        for (int c = 0; c < kC; ++c) sum[c] = 0.f;
+      }
+      const int ch = s4 + 4 * t;
+      const KeyChunk kv = widen8(*reinterpret_cast<const uint4*>(Ks + (ch >> 3) * (kKeys * 128) + sw128_offset(key, (ch & 7) * 8)));
+  #pragma unroll
+      for (int c = 0; c < kC; ++c) sum[c] += sqdiff8(kv, buf[step & 1][c]);
+      if (t == kT - 1) {
+        // transpose-reduce over the group: after the two exchanges lane s holds the total of child s
+        // (and of child s + 4 when C = 8)
+        const bool hi1 = (s4 & 1) != 0, hi2 = (s4 & 2) != 0;
+        float r[kC / 2];
+  #pragma unroll
+        for (int i = 0; i < kC / 2; ++i) {
+          const float send = hi1 ? sum[2 * i] : sum[2 * i + 1];
+          const float keep = hi1 ? sum[2 * i + 1] : sum[2 * i];
+          r[i] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
         }
-      };
-      auto reduce = [&](int bsel, int batch) {
+        float tot[kC / 4];
   #pragma unroll
-        for (int b = 0; b < kKB; ++b) {
-          const int key = warp * 16 + batch * kKB + b;
-          const KeyChunk kv = widen8(*reinterpret_cast<const uint4*>(krow_base + sw128_offset(key, kpos & 63)));
-          float e1 = INFINITY, e2 = INFINITY;
-          int c1 = 0;
+        for (int i = 0; i < kC / 4; ++i) {
+          const float send = hi2 ? r[2 * i] : r[2 * i + 1];
+          const float keep = hi2 ? r[2 * i + 1] : r[2 * i];
+          tot[i] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+        }
+        float e1 = tot[0], e2 = INFINITY;
+        int c1 = s4;
+        if constexpr (kC == 8) {
+          e2 = fmaxf(tot[0], tot[1]);
+          if (tot[1] < tot[0]) { e1 = tot[1]; c1 = s4 + 4; }
+        }
   #pragma unroll
-          for (int t = 0; t < NL; ++t) {
-            float s = sqdiff8(kv, buf[bsel][b][t]);
-  #pragma unroll
-            for (int o = 1; o < kLanesPerChild; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            const int c = t * kChildPerLoad + grp;     // ascending in t: a later equal distance never wins
-            e2 = fminf(e2, fmaxf(s, e1));
-            if (s < e1) { e1 = s; c1 = c; }
-          }
-  #pragma unroll
-          for (int o = kLanesPerChild; o < 32; o <<= 1) {
-            const float b1 = __shfl_xor_sync(0xffffffffu, e1, o);
-            const float b2 = __shfl_xor_sync(0xffffffffu, e2, o);
-            const int cb = __shfl_xor_sync(0xffffffffu, c1, o);
-            e2 = fminf(fmaxf(e1, b1), fminf(e2, b2));
-            if (b1 < e1 || (b1 == e1 && cb < c1)) { e1 = b1; c1 = cb; }
-          }
-          if (lane == 0) {
-            if (done && j0 + key < Nk && C > 1 && !(e2 - e1 > 1e-4f * e2)) {
-              const __nv_bfloat16* Cch = Cc + (head_base + par[key]) * C * D;
-              double best = INFINITY;
-              int bi = 0;
-              for (int c = 0; c < C; ++c) {
-                const double sd = exact_dist_smem<D>(Ks, key, Cch + (size_t)c * D);
-                if (sd < best) { best = sd; bi = c; }
-              }
-              c1 = bi;
+        for (int o = 1; o < 4; o <<= 1) {
+          const float b1 = __shfl_xor_sync(0xffffffffu, e1, o);
+          const float b2 = __shfl_xor_sync(0xffffffffu, e2, o);
+          const int cb = __shfl_xor_sync(0xffffffffu, c1, o);
+          e2 = fminf(fmaxf(e1, b1), fminf(e2, b2));
+          if (b1 < e1 || (b1 == e1 && cb < c1)) { e1 = b1; c1 = cb; }
+        }
+        if (s4 == 0) {
+          if (done && j0 + key < Nk && !(e2 - e1 > 1e-4f * e2)) {
+            const __nv_bfloat16* Cch = Cc + (head_base + par[key]) * kC * D;
+            double best = INFINITY;
+            int bi = 0;
+            for (int c = 0; c < kC; ++c) {
+              const double sd = exact_dist_smem<D>(Ks, key, Cch + (size_t)c * D);
+              if (sd < best) { best = sd; bi = c; }
             }
-            chi[key] = c1;
+            c1 = bi;
           }
+          chi[key] = c1;
         }
-      };
-      issue(0, 0);
-  #pragma unroll
-      for (int batch = 0; batch < kNB; batch += 2) {
-        issue(1, batch + 1);
-        reduce(0, batch);
-        if (batch + 2 < kNB) issue(0, batch + 2);
-        reduce(1, batch + 1);
       }
     }
   }
