@@ -8,10 +8,9 @@
 //            runner-up are closer than the MMA's rounding can separate are all M distances redone in
 //            float64 in the direct form (lowest index wins ties).
 //   child    fp32 direct form sum (k - c)^2 on CUDA cores (2 C d flops per key; a second MMA over all
-//            M C children would cost C times the parent GEMM), float64 recheck for near-ties.  Small
-//            child blocks (C d = 256): the two threads of a key take half of the children each.
-//            Larger ones: four lanes per key, each over a quarter of the head dimension for all C
-//            children (one running sum per child), a transposing butterfly merges the four lanes.
+//            M C children would cost C times the parent GEMM), float64 recheck for near-ties.
+//            Four lanes per key, each over a quarter of the head dimension for all C children of the
+//            key's parent (one running sum per child); a transposing butterfly merges the four lanes.
 #include "avq_tc_common.cuh"
 
 namespace avq {
@@ -21,6 +20,9 @@ using namespace tc;
 
 constexpr int kKeys = 128;
 constexpr int kThreadsA = 256;
+// CTAs per SM the register budget is set for: the d = 64 kernels are small enough (24-48 KB of shared
+// memory, at most 128 TMEM columns up to M = 128) for four (C = 4) or three (C = 8) to share an SM.
+constexpr int assign_min_ctas(int D, int NL) { return D == 64 ? (NL == 1 ? 4 : 3) : 2; }
 
 #ifdef AVQ_PHASE_DEBUG
 __device__ long long g_assign_clocks[64 * 16];
@@ -81,9 +83,8 @@ __device__ double exact_dist_smem(const unsigned char* Ks, int row, const __nv_b
 
 // NL = 16-byte loads per lane that cover one parent's C x d block of children: C * d / 256.
 template <int D, int NL>
-__global__ void __launch_bounds__(kThreadsA, NL == 1 ? 3 : 2)
+__global__ void __launch_bounds__(kThreadsA, assign_min_ctas(D, NL))
 tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmCp,
-                 const __grid_constant__ CUtensorMap tmCc, const int stage_rows_arg,
                  const __nv_bfloat16* __restrict__ Cp, const __nv_bfloat16* __restrict__ Cc,
                  int32_t* __restrict__ pidx, int32_t* __restrict__ cidx, int H, int Nk, int M, int C,
                  uint32_t tmem_cols, int32_t* status_word) {
@@ -93,11 +94,7 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   constexpr int kSub = D / 64;                       // 64-column sub-tiles along the head dimension
   unsigned char* Ks = smem;                          // kSub x [128 x 128 B]
   unsigned char* Cs = Ks + kSub * kKeys * 128;       // kSub x [M x 128 B]
-  const int stage_rows = (NL == 1) ? stage_rows_arg : 0;   // only the small-block variant stages
-  // Small child codebooks (stage_rows = M * C rows of 128 bytes, d = 64 only) are staged whole, so that
-  // the child argmin reads shared memory instead of gathering rows from global memory.
-  unsigned char* Ccs = Cs + kSub * M * 128;          // [stage_rows x 128 B], 128-byte swizzle
-  float* cnorm = reinterpret_cast<float*>(Ccs + stage_rows * 128);   // [M]
+  float* cnorm = reinterpret_cast<float*>(Cs + kSub * M * 128);   // [M]
   float* xd1 = cnorm + M;                            // [2][128] best distance of each column half
   float* xd2 = xd1 + 2 * kKeys;                      // [2][128] runner-up
   float* xkn = xd2 + 2 * kKeys;                      // [2][128] halves of ||k||^2
@@ -120,15 +117,12 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   if (tid == 0) {
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmCp);
-    if (stage_rows) prefetch_tmap(&tmCc);
     mbar_init(&bars[0], 1);
     mbar_init(&bars[1], 1);
     mbar_fence_init();
     *abort_flag = 0;
     *cmax_bits = 0;
-    mbar_expect_tx(&bars[0], (uint32_t)(kSub * (kKeys + M) * 128 + stage_rows * 128));
-    for (int b0 = 0; b0 < stage_rows; b0 += 256)
-      tma_load_2d(Ccs + b0 * 128, &tmCc, 0, h * M * C + b0, &bars[0]);
+    mbar_expect_tx(&bars[0], (uint32_t)(kSub * (kKeys + M) * 128));
 #pragma unroll
     for (int s = 0; s < kSub; ++s) {
       tma_load_3d(Ks + s * kKeys * 128, &tmK, s * 64, j0, bh, &bars[0]);
@@ -257,57 +251,7 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   __syncthreads();
   APHASE(8);
 
-  if constexpr (NL == 1) {
-    // ---- child argmin: the two threads of a key take half of the C children each (fp32 direct form),
-    // eight 16-byte loads in flight per thread; the halves are merged like the parents'
-    {
-      const int a = par[r];
-      const int CH = C >> 1;                           // children per thread (C is 4 or 8)
-      const __nv_bfloat16* Cch = Cc + (((size_t)h * M + a) * C + (size_t)hf * CH) * D;
-      float e1 = INFINITY, e2 = INFINITY;
-      int c1 = 0;
-      for (int c = 0; c < CH; ++c) {
-        const uint4* src = reinterpret_cast<const uint4*>(Cch + (size_t)c * D);
-        float s = 0.f;
-  #pragma unroll
-        for (int g = 0; g < D / 64; ++g) {             // 8 chunks (64 elements) at a time
-          uint4 cv[8];
-  #pragma unroll
-          for (int t = 0; t < 8; ++t)
-            cv[t] = stage_rows ? *reinterpret_cast<const uint4*>(Ccs + sw128_offset(a * C + hf * CH + c, t * 8))
-                               : __ldg(src + g * 8 + t);
-  #pragma unroll
-          for (int t = 0; t < 8; ++t) {
-            const uint4 kv = *reinterpret_cast<const uint4*>(Ks + g * kKeys * 128 + sw128_offset(r, t * 8));
-            s += sqdiff8(kv, cv[t]);
-          }
-        }
-        e2 = fminf(e2, fmaxf(s, e1));
-        if (s < e1) { e1 = s; c1 = hf * CH + c; }
-      }
-      xd1[hf * kKeys + r] = e1;
-      xd2[hf * kKeys + r] = e2;
-      xi1[hf * kKeys + r] = c1;
-    }
-    __syncthreads();
-    if (hf == 0) {
-      const float a1 = xd1[r], a2 = xd2[r], b1 = xd1[kKeys + r], b2 = xd2[kKeys + r];
-      int c1 = (b1 < a1) ? xi1[kKeys + r] : xi1[r];
-      const float e1 = fminf(a1, b1);
-      const float e2 = fminf(fmaxf(a1, b1), fminf(a2, b2));
-      if (done && j0 + r < Nk && !(e2 - e1 > 1e-4f * e2)) {
-        const __nv_bfloat16* Cch = Cc + ((size_t)h * M + par[r]) * C * D;
-        double best = INFINITY;
-        int bi = 0;
-        for (int c = 0; c < C; ++c) {
-          const double s = exact_dist_smem<D>(Ks, r, Cch + (size_t)c * D);
-          if (s < best) { best = s; bi = c; }
-        }
-        c1 = bi;
-      }
-      chi[r] = c1;
-    }
-  } else {
+  {
     // ---- child argmin, four lanes per key: a warp takes 8 keys at a time (two passes over its 16 keys).
     // Lane s of a key's group covers the 16-byte chunks s, s + 4, ... of the key row and of each of the
     // parent's C children (the group reads 64 contiguous bytes of a child row per load), keeps one running
@@ -407,16 +351,8 @@ uint32_t pow2_cols(int n) {
 template <int D, int NL>
 avq_status launch(const avq_problem& p, const void* K, const void* Cp, const void* Cc, int32_t* pidx,
                   int32_t* cidx, int32_t* status_word, cudaStream_t st) {
-  CUtensorMap tmK, tmCp, tmCc;
+  CUtensorMap tmK, tmCp;
   const uint64_t BH = (uint64_t)p.B * p.H;
-  // stage the head's whole child codebook when it is small (d = 64, C = 4, at most 512 rows = 64 KB)
-  const int stage_rows = (NL == 1 && p.M * p.C <= 512) ? p.M * p.C : 0;
-  {
-    const uint64_t dims[2] = {(uint64_t)D, (uint64_t)p.H * p.M * p.C};
-    const uint32_t box[2] = {64, (uint32_t)(stage_rows > 256 ? 256 : (stage_rows ? stage_rows : 8))};
-    avq_status s = make_tmap_bf16(&tmCc, Cc, 2, dims, box);
-    if (s != AVQ_OK) return s;
-  }
   {
     const uint64_t dims[3] = {(uint64_t)D, (uint64_t)p.Nk, BH};
     const uint32_t box[3] = {64, (uint32_t)kKeys, 1};
@@ -429,7 +365,7 @@ avq_status launch(const avq_problem& p, const void* K, const void* Cp, const voi
     avq_status s = make_tmap_bf16(&tmCp, Cp, 2, dims, box);
     if (s != AVQ_OK) return s;
   }
-  const size_t smem = (size_t)(D / 64) * (kKeys + p.M) * 128 + (size_t)stage_rows * 128 +
+  const size_t smem = (size_t)(D / 64) * (kKeys + p.M) * 128 +
                       sizeof(float) * (p.M + 6 * kKeys) +
                       sizeof(int) * (4 * kKeys) + 64 + 1024;
   auto kern = tc_assign_kernel<D, NL>;
@@ -443,7 +379,7 @@ avq_status launch(const avq_problem& p, const void* K, const void* Cp, const voi
     if (dev >= 0 && dev < 64) configured[dev] = smem;
   }
   dim3 grid((p.Nk + kKeys - 1) / kKeys, (unsigned)BH);
-  kern<<<grid, kThreadsA, smem, st>>>(tmK, tmCp, tmCc, stage_rows, static_cast<const __nv_bfloat16*>(Cp),
+  kern<<<grid, kThreadsA, smem, st>>>(tmK, tmCp, static_cast<const __nv_bfloat16*>(Cp),
                                       static_cast<const __nv_bfloat16*>(Cc), pidx, cidx, p.H, p.Nk, p.M, p.C,
                                       pow2_cols(p.M), status_word);
   return cuda_ok(cudaGetLastError());
