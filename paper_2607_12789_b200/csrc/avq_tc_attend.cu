@@ -265,14 +265,17 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       float s[16];
       tmem_ld16(t_s + c0, s);
       const float4* b4 = reinterpret_cast<const float4*>(bias + colbase + c0);
+      // the biased logit stays in the register: an empty parent's -inf becomes a weight of exactly 0
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const float4 b = b4[u];
-        mx = fmaxf(mx, fmaxf(s[4 * u] + b.x, s[4 * u + 1] + b.y));
-        mx = fmaxf(mx, fmaxf(s[4 * u + 2] + b.z, s[4 * u + 3] + b.w));
+        a[c0 + 4 * u] = s[4 * u] + b.x;
+        a[c0 + 4 * u + 1] = s[4 * u + 1] + b.y;
+        a[c0 + 4 * u + 2] = s[4 * u + 2] + b.z;
+        a[c0 + 4 * u + 3] = s[4 * u + 3] + b.w;
+        mx = fmaxf(mx, fmaxf(a[c0 + 4 * u], a[c0 + 4 * u + 1]));
+        mx = fmaxf(mx, fmaxf(a[c0 + 4 * u + 2], a[c0 + 4 * u + 3]));
       }
-#pragma unroll
-      for (int e = 0; e < 16; ++e) a[c0 + e] = s[e];
     } else {
 #pragma unroll
       for (int e = 0; e < 16; ++e) a[c0 + e] = 0.f;
@@ -288,8 +291,8 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // m_run is finite: at least one parent holds a key.
   PHASE_MARK(4);
 
-  // ---- fp32 weights; exact denominator of the parent pass.  Empty parents need no zeroing: the clamp
-  // keeps their weight finite and their count and value sum are zero.
+  // ---- fp32 weights; exact denominator of the parent pass.  Empty parents carry a logit of -inf, hence
+  // a weight of exactly zero; every other logit is at most the maximum (up to one rounding).
   float zfull = 0.f;
   {
     const float negm = -m_run;
@@ -300,10 +303,10 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const float4 n = n4[u];
-          a[c0 + 4 * u] = ex2(fminf(fmaf(a[c0 + 4 * u], sc, negm), 0.f));
-          a[c0 + 4 * u + 1] = ex2(fminf(fmaf(a[c0 + 4 * u + 1], sc, negm), 0.f));
-          a[c0 + 4 * u + 2] = ex2(fminf(fmaf(a[c0 + 4 * u + 2], sc, negm), 0.f));
-          a[c0 + 4 * u + 3] = ex2(fminf(fmaf(a[c0 + 4 * u + 3], sc, negm), 0.f));
+          a[c0 + 4 * u] = ex2(fmaf(a[c0 + 4 * u], sc, negm));
+          a[c0 + 4 * u + 1] = ex2(fmaf(a[c0 + 4 * u + 1], sc, negm));
+          a[c0 + 4 * u + 2] = ex2(fmaf(a[c0 + 4 * u + 2], sc, negm));
+          a[c0 + 4 * u + 3] = ex2(fmaf(a[c0 + 4 * u + 3], sc, negm));
           zfull = fmaf(a[c0 + 4 * u], n.x, zfull);
           zfull = fmaf(a[c0 + 4 * u + 1], n.y, zfull);
           zfull = fmaf(a[c0 + 4 * u + 2], n.z, zfull);
@@ -379,16 +382,19 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (j < M) {
         const uint32_t kj = keys[j];
         const int span = M / kT, kb = part * span;
-#pragma unroll 2
+        int g0 = 0, g1 = 0, g2 = 0, g3 = 0;              // four independent counters: no serial add chain
+#pragma unroll 4
         for (int k = kb; k < kb + span; k += 4) {
           const uint4 kk = *reinterpret_cast<const uint4*>(keys + k);
           asm("{\n\t.reg .pred p0, p1, p2, p3;\n\t"
-              "setp.gt.u32 p0, %1, %5;\n\tsetp.gt.u32 p1, %2, %5;\n\t"
-              "setp.gt.u32 p2, %3, %5;\n\tsetp.gt.u32 p3, %4, %5;\n\t"
-              "@p0 add.s32 %0, %0, 1;\n\t@p1 add.s32 %0, %0, 1;\n\t"
-              "@p2 add.s32 %0, %0, 1;\n\t@p3 add.s32 %0, %0, 1;\n\t}"
-              : "+r"(gt) : "r"(kk.x), "r"(kk.y), "r"(kk.z), "r"(kk.w), "r"(kj));
+              "setp.gt.u32 p0, %4, %8;\n\tsetp.gt.u32 p1, %5, %8;\n\t"
+              "setp.gt.u32 p2, %6, %8;\n\tsetp.gt.u32 p3, %7, %8;\n\t"
+              "@p0 add.s32 %0, %0, 1;\n\t@p1 add.s32 %1, %1, 1;\n\t"
+              "@p2 add.s32 %2, %2, 1;\n\t@p3 add.s32 %3, %3, 1;\n\t}"
+              : "+r"(g0), "+r"(g1), "+r"(g2), "+r"(g3)
+              : "r"(kk.x), "r"(kk.y), "r"(kk.z), "r"(kk.w), "r"(kj));
         }
+        gt = (g0 + g1) + (g2 + g3);
       }
       PHASE_MARK(16);
       if (kT == 2) gt += __shfl_xor_sync(0xffffffffu, gt, 1);
