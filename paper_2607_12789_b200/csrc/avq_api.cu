@@ -107,7 +107,7 @@ avq_status avq_assign(const avq_problem* prob, const void* K, const void* Cp, co
   if (!aligned16(K) || !aligned16(Cp) || !aligned16(Cc) || !aligned16(parent_idx) || !aligned16(child_idx))
     return AVQ_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (use_tensor_path(*prob)) return tc_assign(*prob, K, Cp, Cc, parent_idx, child_idx, nullptr, st);
+  if (use_tensor_path(*prob)) return tc_assign(*prob, K, Cp, Cc, parent_idx, child_idx, nullptr, nullptr, 0, st);
   return simt_assign(*prob, K, Cp, Cc, parent_idx, child_idx, st);
 }
 
@@ -181,9 +181,8 @@ avq_status avq_forward(const avq_problem* prob, const void* Q, const void* K, co
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Regions r = carve(workspace, L);
   if (use_tensor_path(p)) {
-    // one memset: status header, leaf sums and leaf counts are adjacent
-    if (cudaMemsetAsync(workspace, 0, L.zero_end, st) != cudaSuccess) return AVQ_ERR_CUDA;
-    s = tc_assign(p, K, Cp, Cc, r.pidx, r.cidx, r.status_word, st);
+    // status header, leaf sums and leaf counts are adjacent: the assign grid clears them on the side
+    s = tc_assign(p, K, Cp, Cc, r.pidx, r.cidx, r.status_word, workspace, L.zero_end, st);
     if (s != AVQ_OK) return s;
     s = tc_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, r.VpT, r.VcT, true, st);
   } else {

@@ -48,8 +48,10 @@ avq_status simt_attend(const avq_problem& p, const void* Q, const void* Cp, cons
                        cudaStream_t st);
 
 // ---- tensor-core kernels (avq_tc_*.cu) ----
+// zero_base / zero_bytes: a region (multiple of 16 bytes, or none) the assign grid clears on the side
 avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const void* Cc,
-                     int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, cudaStream_t st);
+                     int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, void* zero_base,
+                     size_t zero_bytes, cudaStream_t st);
 avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
                         const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc,
                         void* VpT, void* VcT, bool pre_zeroed, cudaStream_t st);

@@ -27,20 +27,13 @@ leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restri
                     const int32_t* __restrict__ cidx, float* __restrict__ Vc, float* __restrict__ nc,
                     int Nk, int M, int C) {
   tc::pdl_launch_dependents();
-  tc::pdl_wait();                                    // the indices come from the kernel before
   const int bh = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int j0 = blockIdx.x * kKeysPerCta + warp * kKeysPerWarp;
-  if (j0 >= Nk) return;
   const size_t kb = (size_t)bh * Nk;
-  int leaf_l = -1;
-  if (lane < kKeysPerWarp && j0 + lane < Nk) {
-    const int a = __ldg(pidx + kb + j0 + lane);
-    const int c = __ldg(cidx + kb + j0 + lane);
-    leaf_l = a * C + c;
-  }
   // Every lane adds four floats with one 16-byte reduction: a full warp covers a 128-wide row, a
-  // half warp a 64-wide one (two keys per step).
+  // half warp a 64-wide one (two keys per step).  The value rows are the caller's: their loads go out
+  // before the wait for the kernel that writes the indices.
   constexpr int kLanesPerRow = D / 4;
   constexpr int kRowsPerStep = 32 / kLanesPerRow;
   constexpr int kSteps = kKeysPerWarp / kRowsPerStep;
@@ -51,6 +44,14 @@ leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restri
     const int j = j0 + t * kRowsPerStep + sub;
     v[t] = make_uint2(0u, 0u);
     if (j < Nk) v[t] = __ldg(reinterpret_cast<const uint2*>(V + (kb + j) * D) + col);
+  }
+  tc::pdl_wait();                                    // the indices come from the kernel before
+  if (j0 >= Nk) return;
+  int leaf_l = -1;
+  if (lane < kKeysPerWarp && j0 + lane < Nk) {
+    const int a = __ldg(pidx + kb + j0 + lane);
+    const int c = __ldg(cidx + kb + j0 + lane);
+    leaf_l = a * C + c;
   }
 #pragma unroll
   for (int t = 0; t < kSteps; ++t) {

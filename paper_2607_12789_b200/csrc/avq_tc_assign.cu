@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(kThreadsA, assign_min_ctas(D, NL))
 tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmCp,
                  const __nv_bfloat16* __restrict__ Cp, const __nv_bfloat16* __restrict__ Cc,
                  int32_t* __restrict__ pidx, int32_t* __restrict__ cidx, int H, int Nk, int M, int C,
-                 uint32_t tmem_cols, int32_t* status_word) {
+                 uint32_t tmem_cols, int32_t* status_word, uint4* __restrict__ zero_base, uint32_t zero_units) {
   // 1024-byte alignment (swizzle atoms) is requested from the launch, not computed from the pointer, so
   // that the compiler keeps every access in the shared address space.
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -114,6 +114,15 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
   APHASE(0);
   pdl_launch_dependents();   // the next kernel of the call may begin its set-up
+  // Inside avq_forward the grid also clears the accumulators of the aggregation that follows (status
+  // header, leaf sums, leaf counts: zero_units 16-byte words), each CTA an equal slice; the stores drain
+  // while the tile loads.  A bounded wait that expires does so long after CTA 0 has cleared the header.
+  if (zero_units) {
+    const uint32_t ncta = gridDim.x * gridDim.y, cta = blockIdx.y * gridDim.x + blockIdx.x;
+    const uint32_t per = (zero_units + ncta - 1) / ncta;
+    const uint32_t u0 = cta * per, u1 = min(zero_units, u0 + per);
+    for (uint32_t u = u0 + tid; u < u1; u += kThreadsA) zero_base[u] = make_uint4(0u, 0u, 0u, 0u);
+  }
   if (tid == 0) {
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmCp);
@@ -350,7 +359,7 @@ uint32_t pow2_cols(int n) {
 
 template <int D, int NL>
 avq_status launch(const avq_problem& p, const void* K, const void* Cp, const void* Cc, int32_t* pidx,
-                  int32_t* cidx, int32_t* status_word, cudaStream_t st) {
+                  int32_t* cidx, int32_t* status_word, void* zero_base, size_t zero_bytes, cudaStream_t st) {
   CUtensorMap tmK, tmCp;
   const uint64_t BH = (uint64_t)p.B * p.H;
   {
@@ -381,7 +390,8 @@ avq_status launch(const avq_problem& p, const void* K, const void* Cp, const voi
   dim3 grid((p.Nk + kKeys - 1) / kKeys, (unsigned)BH);
   kern<<<grid, kThreadsA, smem, st>>>(tmK, tmCp, static_cast<const __nv_bfloat16*>(Cp),
                                       static_cast<const __nv_bfloat16*>(Cc), pidx, cidx, p.H, p.Nk, p.M, p.C,
-                                      pow2_cols(p.M), status_word);
+                                      pow2_cols(p.M), status_word, static_cast<uint4*>(zero_base),
+                                      (uint32_t)(zero_bytes / 16));
   return cuda_ok(cudaGetLastError());
 }
 
@@ -394,12 +404,14 @@ extern "C" __attribute__((visibility("default"))) int avq_debug_assign_clocks(lo
 #endif
 
 avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const void* Cc,
-                     int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, cudaStream_t st) {
+                     int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, void* zero_base,
+                     size_t zero_bytes, cudaStream_t st) {
+  if (zero_bytes % 16 != 0 || (zero_bytes / 16) >> 31) return AVQ_ERR_WORKSPACE;
   if (p.d == 64)
-    return p.C == 4 ? launch<64, 1>(p, K, Cp, Cc, parent_idx, child_idx, status_word, st)
-                    : launch<64, 2>(p, K, Cp, Cc, parent_idx, child_idx, status_word, st);
-  return p.C == 4 ? launch<128, 2>(p, K, Cp, Cc, parent_idx, child_idx, status_word, st)
-                  : launch<128, 4>(p, K, Cp, Cc, parent_idx, child_idx, status_word, st);
+    return p.C == 4 ? launch<64, 1>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st)
+                    : launch<64, 2>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st);
+  return p.C == 4 ? launch<128, 2>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st)
+                  : launch<128, 4>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st);
 }
 
 }  // namespace avq
