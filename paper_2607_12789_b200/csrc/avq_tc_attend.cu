@@ -98,19 +98,20 @@ __device__ __forceinline__ float store_weights16(unsigned char* A, int r, int co
                                                  const float (&a)[16]) {
   const float4* n4 = reinterpret_cast<const float4*>(cnt16);
   uint32_t pk[8];
-  float z = 0.f;
+  float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;         // independent partial sums: no 16-deep FMA chain
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
     const float4 n = n4[u];
     const uint32_t p0 = pack_bf16(a[4 * u], a[4 * u + 1]);
     const uint32_t p1 = pack_bf16(a[4 * u + 2], a[4 * u + 3]);
-    z = fmaf(__uint_as_float(p0 << 16), n.x, z);
-    z = fmaf(__uint_as_float(p0 & 0xFFFF0000u), n.y, z);
-    z = fmaf(__uint_as_float(p1 << 16), n.z, z);
-    z = fmaf(__uint_as_float(p1 & 0xFFFF0000u), n.w, z);
+    z0 = fmaf(__uint_as_float(p0 << 16), n.x, z0);
+    z1 = fmaf(__uint_as_float(p0 & 0xFFFF0000u), n.y, z1);
+    z2 = fmaf(__uint_as_float(p1 << 16), n.z, z2);
+    z3 = fmaf(__uint_as_float(p1 & 0xFFFF0000u), n.w, z3);
     pk[2 * u] = p0;
     pk[2 * u + 1] = p1;
   }
+  const float z = (z0 + z1) + (z2 + z3);
   unsigned char* sub = A + (col0 >> 6) * (kRows * 128);
   *reinterpret_cast<uint4*>(sub + sw128_offset(r, col0 & 63)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
   *reinterpret_cast<uint4*>(sub + sw128_offset(r, (col0 & 63) + 8)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
@@ -144,8 +145,8 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   unsigned char* CC = Vs + subA * D * 128;               // kSubD x [CHW x 128 B] gathered child codes
   float* cnt = reinterpret_cast<float*>(CC + CHW * D * 2);   // [CT] key counts of the parents
   float* bias = cnt + CT;                                // [CT] 0 for non-empty parents, -inf for empty
-  float* keep = bias + CT;                               // [CT] 0 for parents selected for refinement, else 1
-  float* cntc = keep + CT;                               // [CHW] key counts of the child chunk
+  float* cntk = bias + CT;                               // [CT] key counts with the refined parents' zeroed
+  float* cntc = cntk + CT;                               // [CHW] key counts of the child chunk
   float* biasc = cntc + CHW;                             // [CHW]
   float* w = biasc + CHW;                                // [256] importance
   float* wpart = w + 256;                                // [4][CT]
@@ -233,7 +234,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const float n = j < M ? p.np_[(size_t)bh * M + j] : 0.f;
     cnt[j] = n;
     bias[j] = n > 0.f ? 0.f : -INFINITY;
-    keep[j] = 1.f;
+    cntk[j] = n;
   }
   __syncthreads();
   if (early_exit) {
@@ -258,7 +259,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // This thread's QW (<= 64) parent logits are read from TMEM once and stay in registers through the
   // maximum, the exponentials, the importance sums and the conversion to bf16.
   float a[QW];
-  float mx = -INFINITY;
+  float mx = -INFINITY, mx2 = -INFINITY;
 #pragma unroll
   for (int c0 = 0; c0 < QW; c0 += 16) {
     if (c0 < my_cols) {                                  // warp-uniform
@@ -274,14 +275,14 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         a[c0 + 4 * u + 2] = s[4 * u + 2] + b.z;
         a[c0 + 4 * u + 3] = s[4 * u + 3] + b.w;
         mx = fmaxf(mx, fmaxf(a[c0 + 4 * u], a[c0 + 4 * u + 1]));
-        mx = fmaxf(mx, fmaxf(a[c0 + 4 * u + 2], a[c0 + 4 * u + 3]));
+        mx2 = fmaxf(mx2, fmaxf(a[c0 + 4 * u + 2], a[c0 + 4 * u + 3]));
       }
     } else {
 #pragma unroll
       for (int e = 0; e < 16; ++e) a[c0 + e] = 0.f;
     }
   }
-  float m_run = mx * sc;                                // scale > 0: the maximum commutes with it
+  float m_run = fmaxf(mx, mx2) * sc;                    // scale > 0: the maximum commutes with it
   if (NQ > 1) {
     xm[cq * kRows + r] = m_run;
     row_sync<NQ>(q);
@@ -295,6 +296,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // a weight of exactly zero; every other logit is at most the maximum (up to one rounding).
   float zfull = 0.f;
   {
+    float zf0 = 0.f, zf1 = 0.f, zf2 = 0.f, zf3 = 0.f;
     const float negm = -m_run;
 #pragma unroll
     for (int c0 = 0; c0 < QW; c0 += 16) {
@@ -307,13 +309,14 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           a[c0 + 4 * u + 1] = ex2(fmaf(a[c0 + 4 * u + 1], sc, negm));
           a[c0 + 4 * u + 2] = ex2(fmaf(a[c0 + 4 * u + 2], sc, negm));
           a[c0 + 4 * u + 3] = ex2(fmaf(a[c0 + 4 * u + 3], sc, negm));
-          zfull = fmaf(a[c0 + 4 * u], n.x, zfull);
-          zfull = fmaf(a[c0 + 4 * u + 1], n.y, zfull);
-          zfull = fmaf(a[c0 + 4 * u + 2], n.z, zfull);
-          zfull = fmaf(a[c0 + 4 * u + 3], n.w, zfull);
+          zf0 = fmaf(a[c0 + 4 * u], n.x, zf0);
+          zf1 = fmaf(a[c0 + 4 * u + 1], n.y, zf1);
+          zf2 = fmaf(a[c0 + 4 * u + 2], n.z, zf2);
+          zf3 = fmaf(a[c0 + 4 * u + 3], n.w, zf3);
         }
       }
     }
+    zfull = (zf0 + zf1) + (zf2 + zf3);
     if (NQ > 1) {
       xz[cq * kRows + r] = zfull;
       row_sync<NQ>(q);
@@ -426,7 +429,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       int pos = __popc(bal & ((1u << lane) - 1u));
       for (int u = 0; u < warp; ++u) pos += __popc(wmask[u]);
       sel_list[pos] = j;
-      keep[j] = 0.f;
+      cntk[j] = 0.f;
       if (p.topp_out) p.topp_out[((size_t)bh * p.nblk + blk) * P + pos] = j;
     }
   }
@@ -461,23 +464,24 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   };
   gather_codes(0);
 
-  // ---- masked bf16 weights into shared memory (over the dead codebook) + their denominator
+  // ---- bf16 weights into shared memory (over the dead codebook) + their denominator.  A refined parent
+  // is removed from the numerator by clearing its column of the value tile and from the denominator by
+  // its zeroed count, so the weights themselves need no mask.
+  mbar_wait(bar_ld1, 0, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);   // value sums have landed
+  for (int u = tid; u < (min(P, M) << kLogD); u += kThreads) {
+    const int col = sel_list[u >> kLogD], k = u & (D - 1);
+    *reinterpret_cast<__nv_bfloat16*>(Vs + (col >> 6) * (D * 128) + sw128_offset(k, col & 63)) =
+        __float2bfloat16_rn(0.f);
+  }
   {
     float zloc = 0.f;
 #pragma unroll
     for (int c0 = 0; c0 < QW; c0 += 16) {
       if (c0 < my_cols) {
         float am[16];
-        const float4* k4 = reinterpret_cast<const float4*>(keep + colbase + c0);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const float4 kk = k4[u];
-          am[4 * u] = a[c0 + 4 * u] * kk.x;
-          am[4 * u + 1] = a[c0 + 4 * u + 1] * kk.y;
-          am[4 * u + 2] = a[c0 + 4 * u + 2] * kk.z;
-          am[4 * u + 3] = a[c0 + 4 * u + 3] * kk.w;
-        }
-        zloc += store_weights16(CA, r, colbase + c0, cnt + colbase + c0, am);
+        for (int e = 0; e < 16; ++e) am[e] = a[c0 + e];
+        zloc += store_weights16(CA, r, colbase + c0, cntk + colbase + c0, am);
       }
     }
     xz2[cq * kRows + r] = zloc;
