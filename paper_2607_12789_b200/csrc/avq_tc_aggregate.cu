@@ -76,7 +76,10 @@ constexpr int kSortThreads = 512;
 constexpr int kSortKeysPerThread = 16;
 constexpr int kSortMaxKeys = kSortThreads * kSortKeysPerThread;   // keys per CTA (16-bit key field of the order list)
 constexpr int kSortMaxLeaves = 2048;                              // M * C <= 256 * 8
-constexpr int kSortRatio = 2;                                     // chunked variant from this many keys per leaf
+// The chunked variant is chosen for heads of at least kSortMinKeys keys when a CTA's chunk holds at least
+// 0.8 keys per leaf (measured: faster from there on; short heads leave its 512-thread CTAs idle).
+constexpr int kSortRatio10 = 8;
+constexpr int kSortMinKeys = 2048;
 
 template <int D>
 __global__ void __launch_bounds__(kSortThreads, 2)
@@ -246,7 +249,7 @@ avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const i
   }
   // `pre_zeroed` marks the chained call from avq_forward: the kernel before in the stream is the assign
   // kernel, so the scatter may be launched as its programmatic dependent.
-  // Chunked variant when a CTA's share of a head holds several keys per leaf: about two CTAs per SM.
+  // Chunked variant when a CTA's share of a long head holds about a key per leaf or more: two CTAs per SM.
   const int L = p.M * C;
   int sms = 148;
   {
@@ -264,7 +267,7 @@ avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const i
   int chunk = (p.Nk + per_head - 1) / per_head;
   if (chunk > kSortMaxKeys) chunk = kSortMaxKeys;
   chunk = (chunk + 31) & ~31;
-  if (L <= kSortMaxLeaves && chunk >= kSortRatio * L) {
+  if (L <= kSortMaxLeaves && p.Nk >= kSortMinKeys && chunk * 10 >= kSortRatio10 * L) {
     dim3 g1((p.Nk + chunk - 1) / chunk, BH);
     const size_t smem = sizeof(int) * (2 * (size_t)L + 16) + sizeof(uint32_t) * (size_t)chunk;
     // above the default limit only for the largest leaf count and chunk: opt in once per device
