@@ -565,13 +565,18 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         mxc = fmaxf(mxc, fmaxf(s[4 * u + 2] + b.z, s[4 * u + 3] + b.w));
       }
     }
-    float m_new = fmaxf(m_run, mxc * sc);
+    float m_c = mxc * sc;
     if (NQ > 1) {
-      xm[cq * kRows + r] = mxc * sc;
+      xm[cq * kRows + r] = m_c;
       row_sync<NQ>(q);
 #pragma unroll
-      for (int u = 0; u < NQ; ++u) m_new = fmaxf(m_new, xm[u * kRows + r]);
+      for (int u = 0; u < NQ; ++u) m_c = fmaxf(m_c, xm[u * kRows + r]);
     }
+    // Any reference value works as long as numerator and denominator share it.  The running one is
+    // kept unless the children exceed it by more than 2^kLazyLog2 (weights up to that factor above 1 are
+    // harmless in fp32 and bf16), which spares most rows the rescaling of O and z.
+    constexpr float kLazyLog2 = 8.f;
+    const float m_new = (m_c > m_run + kLazyLog2) ? m_c : m_run;
     const float negm = -m_new;
     if (e0 == 0) PHASE_MARK(14);
     // ---- rescale what has been accumulated if this row's maximum moved
@@ -595,7 +600,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         float a[16];
         tmem_ld16(t_sc + c0, a);
 #pragma unroll
-        for (int e = 0; e < 16; ++e) a[e] = ex2(fminf(fmaf(a[e], sc, negm), 0.f));
+        for (int e = 0; e < 16; ++e) a[e] = ex2(fminf(fmaf(a[e], sc, negm), kLazyLog2));   // clamp: empty children
         zloc += store_weights16(CA, r, cq * QWC + c0, cntc + cq * QWC + c0, a);
       }
       xz2[cq * kRows + r] = zloc;
