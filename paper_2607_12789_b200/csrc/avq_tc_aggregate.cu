@@ -163,30 +163,38 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
     else atomicAdd(reinterpret_cast<float4*>(dst) + lane, make_float4(acc[0], acc[1], acc[2], acc[3]));
     acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
   };
-  for (int i = s0; i < s1; i += kBatch) {
-    uint32_t e[kBatch];
+  auto add_row = [&](uint32_t e, const Word& w) {
+    const int leaf = (int)(e >> 16);
+    if (leaf != cur) { flush(); cur = leaf; }          // warp-uniform
+    if constexpr (D == 64) {
+      acc[0] += __uint_as_float(w << 16);
+      acc[1] += __uint_as_float(w & 0xFFFF0000u);
+    } else {
+      acc[0] += __uint_as_float(w.x << 16);
+      acc[1] += __uint_as_float(w.x & 0xFFFF0000u);
+      acc[2] += __uint_as_float(w.y << 16);
+      acc[3] += __uint_as_float(w.y & 0xFFFF0000u);
+    }
+  };
+  int i = s0;
+  for (; i + kBatch <= s1; i += kBatch) {               // full batches: one list read per batch, no guards
+    const uint32_t ev = order[i + (lane & (kBatch - 1))];
     Word w[kBatch];
 #pragma unroll
-    for (int u = 0; u < kBatch; ++u) {
-      e[u] = order[min(i + u, s1 - 1)];
-      w[u] = __ldg(Vw + (size_t)(e[u] & 0xFFFFu) * 32);
-    }
+    for (int u = 0; u < kBatch; ++u)
+      w[u] = __ldg(Vw + (size_t)(__shfl_sync(0xffffffffu, ev, u) & 0xFFFFu) * 32);
 #pragma unroll
-    for (int u = 0; u < kBatch; ++u) {
-      if (i + u < s1) {                                // warp-uniform
-        const int leaf = (int)(e[u] >> 16);
-        if (leaf != cur) { flush(); cur = leaf; }
-        if constexpr (D == 64) {
-          acc[0] += __uint_as_float(w[u] << 16);
-          acc[1] += __uint_as_float(w[u] & 0xFFFF0000u);
-        } else {
-          acc[0] += __uint_as_float(w[u].x << 16);
-          acc[1] += __uint_as_float(w[u].x & 0xFFFF0000u);
-          acc[2] += __uint_as_float(w[u].y << 16);
-          acc[3] += __uint_as_float(w[u].y & 0xFFFF0000u);
-        }
-      }
-    }
+    for (int u = 0; u < kBatch; ++u) add_row(__shfl_sync(0xffffffffu, ev, u), w[u]);
+  }
+  if (i < s1) {                                         // ragged tail of the share
+    const uint32_t ev = order[min(i + (lane & (kBatch - 1)), s1 - 1)];
+    Word w[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u)
+      w[u] = __ldg(Vw + (size_t)(__shfl_sync(0xffffffffu, ev, u) & 0xFFFFu) * 32);
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u)
+      if (i + u < s1) add_row(__shfl_sync(0xffffffffu, ev, u), w[u]);
   }
   flush();
 }
