@@ -38,6 +38,14 @@ if ROOT not in sys.path:
 import numpy as np
 
 METRIC = "avq_attn_fwd_query_tokens_per_s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of each stage's kernel(s), from the ncu captures
+# summarised under profiles/ (tc_attend_c1.md, tc_attend_c3.md, tc_assign_c3.md); other workloads: None.
+NCU_TRAFFIC = {
+    ("c1_vitb", "assign"): 13.12e6, ("c1_vitb", "aggregate"): 17.67e6 + 6.40e6, ("c1_vitb", "attend"): 14.80e6,
+    ("c3_long", "assign"): 71.59e6 + 3.16e6, ("c3_long", "aggregate"): 75.16e6 + 1.39e6 + 8.46e6,
+    ("c3_long", "attend"): 71.52e6 + 31.00e6,
+}
 UNIT = "query-tokens/s"
 
 
@@ -366,7 +374,7 @@ def main():
     value = job_value(wl, world, ms)
     dom = max(res["stages_ms"], key=res["stages_ms"].get)
     rl = roof(stage_model[dom], pk, res["stages_ms"][dom], wl.dtype)
-    rl.update(kernel=dom, traffic=None, peak_source=pk["source"],
+    rl.update(kernel=dom, traffic=NCU_TRAFFIC.get((wl.name, dom)), peak_source=pk["source"],
               bytes_per_launch=stage_model[dom]["bytes"], flops_per_launch=stage_model[dom]["flops"],
               ms_per_launch=res["stages_ms"][dom])
     fr = roof(fwd_model, pk, ms, wl.dtype)
