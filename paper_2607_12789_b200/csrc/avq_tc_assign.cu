@@ -138,7 +138,7 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       tma_load_2d(Cs + s * M * 128, &tmCp, s * 64, h * M, &bars[0]);
     }
   }
-  if (warp == 0) {
+  if (warp == 1) {                                   // not the warp whose lane 0 is busy issuing the loads
     tmem_alloc(tmem_slot, tmem_cols);
     tmem_relinquish();
   }
@@ -232,7 +232,7 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   APHASE(6);
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_base, tmem_cols);
+  if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
   APHASE(7);
 
   // ---- merge the halves (the lower half holds the lower indices, so it wins ties); recheck near-ties

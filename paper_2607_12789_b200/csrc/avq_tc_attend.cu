@@ -193,7 +193,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       tma_load_2d(CA + s * M * 128, &tmCp, s * 64, h * M, bar_ld0);
     }
   }
-  if (warp == 0) {
+  if (warp == 1) {                                   // not the warp whose lane 0 is busy issuing the loads
     tmem_alloc(tmem_slot, p.tmem_cols);
     tmem_relinquish();
   }
@@ -243,7 +243,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     mbar_wait(bar_ld1, 0, abort_flag, nullptr, 0);
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+    if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
     return;
   }
   uint32_t ph_s = 0, ph_pv = 0;
@@ -674,7 +674,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     tma_store_commit_and_wait_read();
   }
   PHASE_MARK(28);
-  if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+  if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
   PHASE_MARK(29);
 }
 
