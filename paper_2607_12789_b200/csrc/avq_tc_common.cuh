@@ -76,21 +76,32 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: polls without blocking, looks at the clock every few polls, gives up after
-// kWaitLimitNs or kWaitLimitPolls.  Returns false (and flags the failure) when it gives up or
-// when the CTA has already aborted.
-constexpr uint32_t kWaitLimitPolls = 1u << 24;
+// Phase test that may suspend the warp in hardware for up to about `hint_ns` before it answers: a waiting
+// warp then takes no issue slots from the warps (of this or another CTA on the SM) that have work.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: each try suspends for a few microseconds at most; after every failed try the abort flag
+// and the clock are looked at; gives up after kWaitLimitNs or kWaitLimitPolls tries.  Returns false (and
+// flags the failure) when it gives up or when the CTA has already aborted.
+constexpr uint32_t kWaitLimitPolls = 1u << 22;
+constexpr uint32_t kWaitTryNs = 4000;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                           int32_t* status_word, int32_t code) {
   if (mbar_test_wait(bar, parity)) return true;
   const unsigned long long t0 = global_timer_ns();
-  for (uint32_t polls = 1; polls < kWaitLimitPolls; ++polls) {
-    if (mbar_test_wait(bar, parity)) return true;
-    if ((polls & 7u) == 0) {
-      if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) break;
-      __nanosleep(32);
-    }
+  for (uint32_t polls = 0; polls < kWaitLimitPolls; ++polls) {
+    if (mbar_try_wait(bar, parity, kWaitTryNs)) return true;
+    if (*abort_flag) return false;
+    if (global_timer_ns() - t0 > kWaitLimitNs) break;
   }
   *abort_flag = 1;
   if (status_word) atomicCAS(status_word, 0, code);
