@@ -200,7 +200,7 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
 }
 
 // One CTA: 8 consecutive parents of one (batch, head); thread k owns head-dimension index k.
-// All loads of four parents are issued before their first use.
+// 32 loads per thread are issued before their first use.
 template <int D, int C>
 __global__ void __launch_bounds__(D)
 finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, float* __restrict__ Vp,
@@ -210,17 +210,18 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
   tc::pdl_wait();                                    // the leaf sums come from the kernel before
   const int bh = blockIdx.y, m0 = blockIdx.x * 8, k = threadIdx.x;
   __align__(16) __nv_bfloat16 pk[8];
+  constexpr int kPer = (C == 4) ? 8 : 4;             // parents whose loads are in flight together (32 floats)
 #pragma unroll
-  for (int g = 0; g < 2; ++g) {
-    float x[4][C];
+  for (int g = 0; g < 8 / kPer; ++g) {
+    float x[kPer][C];
 #pragma unroll
-    for (int mm = 0; mm < 4; ++mm)
+    for (int mm = 0; mm < kPer; ++mm)
 #pragma unroll
       for (int c = 0; c < C; ++c)
-        x[mm][c] = Vc[((((size_t)bh * M + m0 + g * 4 + mm) * C) + c) * D + k];
+        x[mm][c] = Vc[((((size_t)bh * M + m0 + g * kPer + mm) * C) + c) * D + k];
 #pragma unroll
-    for (int mm = 0; mm < 4; ++mm) {
-      const int m = m0 + g * 4 + mm;
+    for (int mm = 0; mm < kPer; ++mm) {
+      const int m = m0 + g * kPer + mm;
       __align__(16) __nv_bfloat16 ck[C];
       float s = 0.f;
 #pragma unroll
@@ -229,7 +230,7 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
         ck[c] = __float2bfloat16_rn(x[mm][c]);
       }
       Vp[((size_t)bh * M + m) * D + k] = s;
-      pk[g * 4 + mm] = __float2bfloat16_rn(s);
+      pk[g * kPer + mm] = __float2bfloat16_rn(s);
       if (VcT) {
         __nv_bfloat16* dst = VcT + (((size_t)bh * M + m) * D + k) * C;
         if (C == 8) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(ck);
