@@ -107,3 +107,32 @@ def test_aggregate_long_heads_few_leaves(H, N, d, M, C):
         scale = 1e-6 * np.sqrt(np.maximum(rnc, 1.0))[..., None] * 50 + 1e-5 * np.abs(rVc)
         assert (np.abs(Vc[0, h].cpu().numpy() - rVc) <= scale + 1e-4).all()
         assert np.allclose(Vp[0, h].cpu().numpy(), rVp, rtol=2e-5, atol=2e-3)
+
+
+def _random_shapes(n, seed):
+    g = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        d = int(g.choice([64, 128]))
+        C = int(g.choice([4, 8]))
+        M = int(g.choice([32, 64, 96, 128, 160, 256]))
+        P = int(g.choice([0, 1, M // 8, M // 4, M]))
+        H = int(g.integers(1, 4))
+        B = int(g.integers(1, 3))
+        N = int(g.integers(129, 1400))
+        out.append(synth.Workload(f"rnd{i}", B=B, H=H, N=N, d=d, M=M, C=C, P=P, block_q=128, seed=500 + i,
+                                  alpha=float(g.choice([0.3, 0.8])), hot_queries=bool(g.integers(0, 2))))
+    return out
+
+
+@pytest.mark.parametrize("wl", _random_shapes(12, seed=20261), ids=lambda w: f"{w.name}-B{w.B}H{w.H}N{w.N}d{w.d}M{w.M}C{w.C}P{w.P}")
+def test_random_shapes_full_parity(wl):
+    """Seeded random shapes inside the tensor-core envelope (ragged lengths, every d, C, several M and P,
+    endpoints included): every stage against the oracle, whole tensors."""
+    parity.full_parity(wl)
+
+
+def test_long_ragged_head_uses_chunked_aggregate_end_to_end():
+    """A ragged long head over few leaves (the chunked aggregate inside avq_forward), sampled against the oracle."""
+    wl = synth.sweep_point(16384, 32, 4).with_(H=2, N=16384 + 77, name="ragged_long")
+    parity.sampled_parity(wl, heads=[(0, 1)], blocks_per_head=4)
