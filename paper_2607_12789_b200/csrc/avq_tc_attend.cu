@@ -131,6 +131,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // that the compiler keeps every access in the shared address space.
   extern __shared__ __align__(1024) unsigned char smem[];
   constexpr int kThreads = 128 * NQ;
+  constexpr int kScLane = kThreads / 2;                  // lane 0 of a warp in the other half of the CTA
   constexpr int kSubD = D / 64;
   constexpr int kLogD = (D == 128) ? 7 : 6;
   constexpr int kLogChunks = kLogD - 3;                  // 16-byte chunks per codeword row
@@ -505,15 +506,18 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                   umma_desc_sw128(va + (k / 4) * D * 128 + (k % 4) * 32), idesc_o, k > 0);
     }
     umma_commit(bar_pv);
-    if (PC > 0) {
-      const uint32_t idesc = umma_idesc_bf16(kRows, np16);
-      const uint32_t qa = smem_u32(Qs), ca = smem_u32(CC);
+  }
+  // The child-score MMAs are issued by a lane of another warp: an issuing lane stalls at the tensor pipe's
+  // pace, and two short stalls side by side delay the next CTA-wide barrier less than one long one.
+  if (tid == kScLane && PC > 0) {
+    tc_fence_after();
+    const uint32_t idesc = umma_idesc_bf16(kRows, np16);
+    const uint32_t qa = smem_u32(Qs), ca = smem_u32(CC);
 #pragma unroll
-      for (int k = 0; k < D / 16; ++k)
-        umma_bf16(tmem_base, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
-                  umma_desc_sw128(ca + (k / 4) * np16 * 128 + (k % 4) * 32), idesc, k > 0);
-      umma_commit(bar_s);
-    }
+    for (int k = 0; k < D / 16; ++k)
+      umma_bf16(tmem_base, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
+                umma_desc_sw128(ca + (k / 4) * np16 * 128 + (k % 4) * 32), idesc, k > 0);
+    umma_commit(bar_s);
   }
 
   // ---- child chunks
@@ -631,7 +635,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       fence_proxy_async();
       tc_fence_before();
       __syncthreads();
-      if (tid == 0) {
+      if (tid == kScLane) {
         tc_fence_after();
         const uint32_t idesc = umma_idesc_bf16(kRows, np16);
         const uint32_t qa = smem_u32(Qs), ca = smem_u32(CC);
