@@ -62,7 +62,6 @@ __device__ __forceinline__ float sqdiff8(const KeyChunk& k, const uint4& c) {
   asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(acc));
   return lo + hi;
 }
-__device__ __forceinline__ float sqdiff8(const uint4& a, const uint4& b) { return sqdiff8(widen8(a), b); }
 
 // element `col` (0..D-1) of key row `row` in the swizzled key tile
 template <int D>
