@@ -136,3 +136,24 @@ def test_long_ragged_head_uses_chunked_aggregate_end_to_end():
     """A ragged long head over few leaves (the chunked aggregate inside avq_forward), sampled against the oracle."""
     wl = synth.sweep_point(16384, 32, 4).with_(H=2, N=16384 + 77, name="ragged_long")
     parity.sampled_parity(wl, heads=[(0, 1)], blocks_per_head=4)
+
+
+def test_degenerate_all_keys_on_one_codeword():
+    """Every key equals one parent codeword: that parent holds all keys, every other parent is empty, the
+    importances are zero but one, and the top-P set is that parent plus the lowest-index empty ones (the
+    tie rule across a whole group of equal importances); empty children must not disturb the maxima."""
+    wl = synth.C1.with_(B=1, H=2, N=512, seed=41)
+    x = synth.generate(wl)
+    for h in range(wl.H):
+        x["K"][0, h, :, :] = x["Cp"][h, 5]
+    rep = parity.full_parity(wl, x=x)
+    assert rep["empty_parents"] == wl.H * (wl.M - 1)
+    assert rep["topp_flips_excused"] == 0
+
+
+def test_single_query_block_shorter_than_a_tile_and_tiny_key_set():
+    """Nq = 1 and Nk = 5: one ragged query tile, one ragged key tile, almost every codeword empty."""
+    wl = synth.C1.with_(B=1, H=1, N=5, seed=43)
+    x = synth.generate(wl)
+    x["Q"] = np.ascontiguousarray(x["Q"][:, :, :1])
+    parity.full_parity(wl, x=x)
