@@ -444,23 +444,31 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   int ncols = min(PC, CHW);
   int np16 = (ncols + 15) & ~15;
   auto gather_codes = [&](int e_first) {
-    // row e (local column) = Cc[h, sel_list[(e_first+e)/C], (e_first+e)%C, :]; padding rows are zero
-    const int total = np16 << kLogChunks;
-    for (int u = tid; u < total; u += kThreads) {
-      const int row = u >> kLogChunks, ch = u & ((1 << kLogChunks) - 1);
-      unsigned char* dst = CC + (ch >> 3) * (np16 * 128) + sw128_offset(row, (ch & 7) * 8);
+    // row e (local column) = Cc[h, sel_list[(e_first+e)/C], (e_first+e)%C, :]; padding rows are zero.
+    // The child counts are fetched first so that their latency hides behind the copies.
+    float n_child = 0.f;
+    if (tid < ncols) {                                   // CHW <= 128 <= kThreads
+      const int e = e_first + tid;
+      n_child = __ldg(ncb + ((size_t)sel_list[e >> logC] << logC) + (e & (C - 1)));
+    }
+    // a thread keeps its 16-byte chunk column and walks down the rows (kThreads is a multiple of the
+    // chunks per row)
+    constexpr int kRowsPerPass = kThreads >> kLogChunks;
+    const int ch = tid & ((1 << kLogChunks) - 1);
+    const uint32_t dst_col = (uint32_t)((ch >> 3) * (np16 * 128));
+    const __nv_bfloat16* src_col = Cch + ch * 8;
+    for (int row = tid >> kLogChunks; row < np16; row += kRowsPerPass) {
+      unsigned char* dst = CC + dst_col + sw128_offset(row, (ch & 7) * 8);
       if (row < ncols) {
         const int e = e_first + row;
-        cp_async16(dst, Cch + (((size_t)sel_list[e >> logC] << logC) + (e & (C - 1))) * D + ch * 8);
+        cp_async16(dst, src_col + (((size_t)sel_list[e >> logC] << logC) + (e & (C - 1))) * D);
       } else {
         *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
       }
     }
-    if (tid < CHW) {                                     // CHW <= 128 <= kThreads
-      const int e = e_first + tid;
-      const float n = tid < ncols ? ncb[((size_t)sel_list[e >> logC] << logC) + (e & (C - 1))] : 0.f;
-      cntc[tid] = n;
-      biasc[tid] = n > 0.f ? 0.f : -INFINITY;
+    if (tid < CHW) {
+      cntc[tid] = n_child;
+      biasc[tid] = n_child > 0.f ? 0.f : -INFINITY;
     }
   };
   gather_codes(0);
