@@ -66,8 +66,8 @@ Layout make_layout(const avq_problem& p, int32_t /*P*/, int32_t /*block_q*/) {
   L.Vp = take(sizeof(float) * BH * p.M * p.d);
   L.np = take(sizeof(float) * BH * p.M);
   if (use_tensor_path(p)) {
-    L.VpT = take(2 * BH * p.M * p.d);
-    L.VcT = take(2 * BH * p.M * p.C * p.d);
+    L.Vpb = take(2 * BH * p.M * p.d);
+    L.Vcb = take(2 * BH * p.M * p.C * p.d);
   }
   L.total = off;
   return L;
@@ -130,7 +130,7 @@ namespace {
 struct Regions {
   int32_t *status_word, *pidx, *cidx;
   float *Vp, *np_, *Vc, *nc;
-  void *VpT, *VcT;
+  void *Vpb, *Vcb;
 };
 Regions carve(void* workspace, const Layout& L) {
   char* ws = static_cast<char*>(workspace);
@@ -142,15 +142,15 @@ Regions carve(void* workspace, const Layout& L) {
   r.np_ = reinterpret_cast<float*>(ws + L.np);
   r.Vc = reinterpret_cast<float*>(ws + L.Vc);
   r.nc = reinterpret_cast<float*>(ws + L.nc);
-  r.VpT = ws + L.VpT;
-  r.VcT = ws + L.VcT;
+  r.Vpb = ws + L.Vpb;
+  r.Vcb = ws + L.Vcb;
   return r;
 }
 avq_status attend_stage(const avq_problem& p, const Regions& r, const void* Q, const void* Cp, const void* Cc,
                         int32_t P, int32_t block_q, void* Y, int32_t* topp_out, float* importance_out,
                         bool chained, cudaStream_t st) {
   if (use_tensor_path(p))
-    return tc_attend(p, Q, Cp, Cc, r.np_, r.nc, r.VpT, r.VcT, P, Y, topp_out, importance_out, r.status_word,
+    return tc_attend(p, Q, Cp, Cc, r.np_, r.nc, r.Vpb, r.Vcb, P, Y, topp_out, importance_out, r.status_word,
                      chained, st);
   return simt_attend(p, Q, Cp, Cc, r.Vp, r.np_, r.Vc, r.nc, P, block_q, Y, topp_out, importance_out, st);
 }
@@ -184,7 +184,7 @@ avq_status avq_forward(const avq_problem* prob, const void* Q, const void* K, co
     // status header, leaf sums and leaf counts are adjacent: the assign grid clears them on the side
     s = tc_assign(p, K, Cp, Cc, r.pidx, r.cidx, r.status_word, workspace, L.zero_end, st);
     if (s != AVQ_OK) return s;
-    s = tc_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, r.VpT, r.VcT, true, st);
+    s = tc_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, r.Vpb, r.Vcb, true, st);
   } else {
     if (cudaMemsetAsync(r.status_word, 0, 256, st) != cudaSuccess) return AVQ_ERR_CUDA;
     s = simt_assign(p, K, Cp, Cc, r.pidx, r.cidx, st);

@@ -19,8 +19,8 @@ struct Layout {
   size_t child_idx = 0;    // int32 [B,H,Nk]
   size_t Vp = 0;           // f32 [B,H,M,d]
   size_t np = 0;           // f32 [B,H,M]
-  size_t VpT = 0;          // bf16 [B,H,d,M]      (tensor-core path only)
-  size_t VcT = 0;          // bf16 [B,H,M,d,C]    (tensor-core path only)
+  size_t Vpb = 0;          // bf16 [B,H,M,d]      copy of Vp (tensor-core path only)
+  size_t Vcb = 0;          // bf16 [B,H,M,C,d]    copy of Vc (tensor-core path only)
   size_t total = 0;
 };
 
@@ -54,9 +54,9 @@ avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const 
                      size_t zero_bytes, cudaStream_t st);
 avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
                         const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc,
-                        void* VpT, void* VcT, bool pre_zeroed, cudaStream_t st);
+                        void* Vpb, void* Vcb, bool pre_zeroed, cudaStream_t st);
 avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc,
-                     const float* np_, const float* nc, const void* VpT, const void* VcT, int32_t P,
+                     const float* np_, const float* nc, const void* Vpb, const void* Vcb, int32_t P,
                      void* Y, int32_t* topp_out, float* importance_out, int32_t* status_word,
                      bool chained, cudaStream_t st);   // chained: launched right behind tc_aggregate
 

@@ -5,9 +5,10 @@
 //                      the leaf's count is bumped.  Only the leaf level is scattered.
 // finalize_kernel      per parent: Vp = sum over its children (every key sits in exactly one
 //                      child, so the parent sum is the sum of its leaves), np likewise, and
-//                      the bf16 operand copies the attention kernel stages with TMA:
-//                        VpT [B,H,d,M]    value sums with the codeword index fastest
-//                        VcT [B,H,M,d,C]  per parent a contiguous d x C block, child fastest
+//                      the bf16 operand copies the attention kernel stages (rows = codewords, the
+//                      MN-major B operand of its value MMAs):
+//                        Vpb [B,H,M,d]    parent value sums
+//                        Vcb [B,H,M,C,d]  leaf value sums: a parent's C children are C consecutive rows
 #include <type_traits>
 
 #include "avq_tc_common.cuh"
@@ -204,12 +205,11 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
 template <int D, int C>
 __global__ void __launch_bounds__(D)
 finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, float* __restrict__ Vp,
-                float* __restrict__ np_, __nv_bfloat16* __restrict__ VpT, __nv_bfloat16* __restrict__ VcT,
+                float* __restrict__ np_, __nv_bfloat16* __restrict__ Vpb, __nv_bfloat16* __restrict__ Vcb,
                 int M) {
   tc::pdl_launch_dependents();
   tc::pdl_wait();                                    // the leaf sums come from the kernel before
   const int bh = blockIdx.y, m0 = blockIdx.x * 8, k = threadIdx.x;
-  __align__(16) __nv_bfloat16 pk[8];
   constexpr int kPer = (C == 4) ? 8 : 4;             // parents whose loads are in flight together (32 floats)
 #pragma unroll
   for (int g = 0; g < 8 / kPer; ++g) {
@@ -221,24 +221,17 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
         x[mm][c] = Vc[((((size_t)bh * M + m0 + g * kPer + mm) * C) + c) * D + k];
 #pragma unroll
     for (int mm = 0; mm < kPer; ++mm) {
-      const int m = m0 + g * kPer + mm;
-      __align__(16) __nv_bfloat16 ck[C];
+      const size_t row = (size_t)bh * M + m0 + g * kPer + mm;
       float s = 0.f;
 #pragma unroll
       for (int c = 0; c < C; ++c) {
         s += x[mm][c];
-        ck[c] = __float2bfloat16_rn(x[mm][c]);
+        if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(x[mm][c]);
       }
-      Vp[((size_t)bh * M + m) * D + k] = s;
-      pk[g * kPer + mm] = __float2bfloat16_rn(s);
-      if (VcT) {
-        __nv_bfloat16* dst = VcT + (((size_t)bh * M + m) * D + k) * C;
-        if (C == 8) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(ck);
-        else *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(ck);
-      }
+      Vp[row * D + k] = s;
+      if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(s);
     }
   }
-  if (VpT) *reinterpret_cast<uint4*>(VpT + ((size_t)bh * D + k) * M + m0) = *reinterpret_cast<const uint4*>(pk);
   if (k < 8) {
     const int m = m0 + k;
     float s = 0.f;
@@ -250,7 +243,7 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
 
 template <int D, int C>
 avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const int32_t* cidx, float* Vp,
-               float* np_, float* Vc, float* nc, void* VpT, void* VcT, bool pre_zeroed, cudaStream_t st) {
+               float* np_, float* Vc, float* nc, void* Vpb, void* Vcb, bool pre_zeroed, cudaStream_t st) {
   const unsigned BH = (unsigned)(p.B * p.H);
   if (!pre_zeroed) {
     if (cudaMemsetAsync(Vc, 0, sizeof(float) * (size_t)BH * p.M * C * D, st) != cudaSuccess) return AVQ_ERR_CUDA;
@@ -301,20 +294,20 @@ avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const i
   }
   dim3 g2(p.M / 8, BH);
   return cuda_ok(tc::launch_pdl(finalize_kernel<D, C>, g2, dim3(D), 0, st, true, static_cast<const float*>(Vc),
-                                static_cast<const float*>(nc), Vp, np_, static_cast<__nv_bfloat16*>(VpT),
-                                static_cast<__nv_bfloat16*>(VcT), p.M));
+                                static_cast<const float*>(nc), Vp, np_, static_cast<__nv_bfloat16*>(Vpb),
+                                static_cast<__nv_bfloat16*>(Vcb), p.M));
 }
 
 }  // namespace
 
 avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
-                        const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc, void* VpT,
-                        void* VcT, bool pre_zeroed, cudaStream_t st) {
+                        const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc, void* Vpb,
+                        void* Vcb, bool pre_zeroed, cudaStream_t st) {
   if (p.d == 64)
-    return p.C == 4 ? run<64, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, VpT, VcT, pre_zeroed, st)
-                    : run<64, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, VpT, VcT, pre_zeroed, st);
-  return p.C == 4 ? run<128, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, VpT, VcT, pre_zeroed, st)
-                  : run<128, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, VpT, VcT, pre_zeroed, st);
+    return p.C == 4 ? run<64, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, st)
+                    : run<64, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, st);
+  return p.C == 4 ? run<128, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, st)
+                  : run<128, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, st);
 }
 
 }  // namespace avq

@@ -37,7 +37,7 @@ constexpr int kRows = 128;
 
 struct AttendParams {
   const __nv_bfloat16* Cc;    // [H, M, C, d]
-  const __nv_bfloat16* VcT;   // [B*H, M, d, C]
+  const __nv_bfloat16* Vcb;   // [B*H, M, C, d]
   const float* np_;           // [B*H, M]
   const float* nc;            // [B*H, M, C]
   __nv_bfloat16* Y;           // [B*H, Nq, d]
@@ -125,7 +125,7 @@ __device__ __forceinline__ float store_weights16(unsigned char* A, int r, int co
 template <int D, int NQ, int CT>
 __global__ void __launch_bounds__(128 * NQ, 4 / NQ)
 tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmCp,
-                 const __grid_constant__ CUtensorMap tmVpT, const __grid_constant__ CUtensorMap tmY,
+                 const __grid_constant__ CUtensorMap tmVpb, const __grid_constant__ CUtensorMap tmY,
                  const AttendParams p) {
   // 1024-byte alignment (swizzle atoms) is requested from the launch, not computed from the pointer, so
   // that the compiler keeps every access in the shared address space.
@@ -142,7 +142,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int M = p.M, C = p.C, P = p.P, logC = p.logC;
   unsigned char* Qs = smem;                              // kSubD x [128 x 128 B]
   unsigned char* CA = Qs + kSubD * kRows * 128;          // parent codes, later the bf16 weights
-  unsigned char* Vs = CA + ca_bytes;                     // subA x [D x 128 B] value sums
+  unsigned char* Vs = CA + ca_bytes;                     // value rows: kSubD x [rows x 128 B], rows = M or a chunk's children
   unsigned char* CC = Vs + subA * D * 128;               // kSubD x [CHW x 128 B] gathered child codes
   float* cnt = reinterpret_cast<float*>(CC + CHW * D * 2);   // [CT] key counts of the parents
   float* bias = cnt + CT;                                // [CT] 0 for non-empty parents, -inf for empty
@@ -180,7 +180,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (tid == 0) {
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmCp);
-    prefetch_tmap(&tmVpT);
+    prefetch_tmap(&tmVpb);
     mbar_init(bar_ld0, 1);
     mbar_init(bar_ld1, 1);
     mbar_init(bar_s, 1);
@@ -206,7 +206,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const uint32_t t_s = t_row + (uint32_t)colbase;
   const uint32_t t_sc = t_row + (uint32_t)(cq * QWC);
   const uint32_t t_o = t_row + (uint32_t)(CT + cq * (D / NQ));
-  const uint32_t idesc_o = umma_idesc_bf16(kRows, D);
+  const uint32_t idesc_o = umma_idesc_bf16(kRows, D) | (1u << 16);   // B (the value rows) is MN-major
   const float sc = p.scale_log2e;
   PHASE_MARK(1);
   if (tid == 0) {
@@ -227,9 +227,9 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (tid == 0) {
     // a wait that expired in an earlier CTA or kernel of this call: do not start more work
     early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
-    const int subM = (M + 63) >> 6;
-    mbar_expect_tx(bar_ld1, (uint32_t)(subM * D * 128));
-    for (int s = 0; s < subM; ++s) tma_load_2d(Vs + s * D * 128, &tmVpT, s * 64, bh * D, bar_ld1);
+    mbar_expect_tx(bar_ld1, (uint32_t)(kSubD * M * 128));
+#pragma unroll
+    for (int s = 0; s < kSubD; ++s) tma_load_2d(Vs + s * M * 128, &tmVpb, s * 64, bh * M, bar_ld1);
   }
   for (int j = tid; j < CT; j += kThreads) {
     const float n = j < M ? p.np_[(size_t)bh * M + j] : 0.f;
@@ -443,22 +443,17 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const float* ncb = p.nc + (size_t)bh * M * C;
   int ncols = min(PC, CHW);
   int np16 = (ncols + 15) & ~15;
-  auto gather_codes = [&](int e_first) {
-    // row e (local column) = Cc[h, sel_list[(e_first+e)/C], (e_first+e)%C, :]; padding rows are zero.
-    // The child counts are fetched first so that their latency hides behind the copies.
-    float n_child = 0.f;
-    if (tid < ncols) {                                   // CHW <= 128 <= kThreads
-      const int e = e_first + tid;
-      n_child = __ldg(ncb + ((size_t)sel_list[e >> logC] << logC) + (e & (C - 1)));
-    }
-    // a thread keeps its 16-byte chunk column and walks down the rows (kThreads is a multiple of the
-    // chunks per row)
+  // Rows of a chunk, gathered into a K-major / row-per-codeword tile of np16 rows (kSubD sub-tiles of 64
+  // columns): local row e = src[sel_list[(e_first+e)/C] * C + (e_first+e)%C, :]; padding rows are zero.
+  // A thread keeps its 16-byte chunk column and walks down the rows (kThreads is a multiple of the chunks
+  // per row).
+  auto gather_rows = [&](unsigned char* tile, const __nv_bfloat16* src, int e_first) {
     constexpr int kRowsPerPass = kThreads >> kLogChunks;
     const int ch = tid & ((1 << kLogChunks) - 1);
     const uint32_t dst_col = (uint32_t)((ch >> 3) * (np16 * 128));
-    const __nv_bfloat16* src_col = Cch + ch * 8;
+    const __nv_bfloat16* src_col = src + ch * 8;
     for (int row = tid >> kLogChunks; row < np16; row += kRowsPerPass) {
-      unsigned char* dst = CC + dst_col + sw128_offset(row, (ch & 7) * 8);
+      unsigned char* dst = tile + dst_col + sw128_offset(row, (ch & 7) * 8);
       if (row < ncols) {
         const int e = e_first + row;
         cp_async16(dst, src_col + (((size_t)sel_list[e >> logC] << logC) + (e & (C - 1))) * D);
@@ -466,6 +461,15 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
       }
     }
+  };
+  auto gather_codes = [&](int e_first) {
+    // the child counts are fetched first so that their latency hides behind the copies
+    float n_child = 0.f;
+    if (tid < ncols) {                                   // CHW <= 128 <= kThreads
+      const int e = e_first + tid;
+      n_child = __ldg(ncb + ((size_t)sel_list[e >> logC] << logC) + (e & (C - 1)));
+    }
+    gather_rows(CC, Cch, e_first);
     if (tid < CHW) {
       cntc[tid] = n_child;
       biasc[tid] = n_child > 0.f ? 0.f : -INFINITY;
@@ -474,13 +478,12 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   gather_codes(0);
 
   // ---- bf16 weights into shared memory (over the dead codebook) + their denominator.  A refined parent
-  // is removed from the numerator by clearing its column of the value tile and from the denominator by
-  // its zeroed count, so the weights themselves need no mask.
+  // is removed from the numerator by clearing its row of the value tile (d / 8 16-byte stores) and from the
+  // denominator by its zeroed count, so the weights themselves need no mask.
   mbar_wait(bar_ld1, 0, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);   // value sums have landed
-  for (int u = tid; u < (min(P, M) << kLogD); u += kThreads) {
-    const int col = sel_list[u >> kLogD], k = u & (D - 1);
-    *reinterpret_cast<__nv_bfloat16*>(Vs + (col >> 6) * (D * 128) + sw128_offset(k, col & 63)) =
-        __float2bfloat16_rn(0.f);
+  for (int u = tid; u < (min(P, M) << kLogChunks); u += kThreads) {
+    const int row = sel_list[u >> kLogChunks], ch = u & ((1 << kLogChunks) - 1);
+    *reinterpret_cast<uint4*>(Vs + (ch >> 3) * (M * 128) + sw128_offset(row, (ch & 7) * 8)) = make_uint4(0, 0, 0, 0);
   }
   {
     float zloc = 0.f;
@@ -511,7 +514,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const uint32_t aa = smem_u32(CA), va = smem_u32(Vs);
       for (int k = 0; k < M / 16; ++k)
         umma_bf16(tmem_base + CT, umma_desc_sw128(aa + (k / 4) * kRows * 128 + (k % 4) * 32),
-                  umma_desc_sw128(va + (k / 4) * D * 128 + (k % 4) * 32), idesc_o, k > 0);
+                  umma_desc_sw128_mn(va + k * 2048, (uint32_t)(M * 128)), idesc_o, k > 0);
     }
     umma_commit(bar_pv);
   }
@@ -529,7 +532,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   }
 
   // ---- child chunks
-  const __nv_bfloat16* Vch = p.VcT + (size_t)bh * M * D * C;
+  const __nv_bfloat16* Vch = p.Vcb + (size_t)bh * M * C * D;
   for (int e0 = 0; e0 < PC; e0 += CHW) {
     // The previous second MMA must have released A and Vs before they are rewritten.
     if (e0 == 0) PHASE_MARK(10);
@@ -537,26 +540,9 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     ph_pv ^= 1;
     tc_fence_after();
     if (e0 == 0) PHASE_MARK(11);
-    // values of this chunk: Vs[k][e] = VcT[bh, parent, k, child]; one parent's C children are contiguous
-    // per k.  Asynchronous copies: they land while the chunk's logits are turned into weights.
-    {
-      const int npar = ncols >> logC, par0 = e0 >> logC;
-      const int vtotal = npar << kLogD;
-      for (int u = tid; u < vtotal; u += kThreads) {
-        const int pr = u >> kLogD, k = u & (D - 1);
-        const __nv_bfloat16* src = Vch + (((size_t)sel_list[par0 + pr] << kLogD) + k) * C;
-        const int col = pr << logC;
-        unsigned char* dst = Vs + (col >> 6) * (D * 128) + sw128_offset(k, col & 63);
-        if (C == 8) cp_async16(dst, src);
-        else cp_async8(dst, src);
-      }
-    }
-    // zero the padding columns [ncols, np16) of the value tile (they meet finite weights; 0 * NaN is NaN)
-    for (int u = tid; u < ((np16 - ncols) << kLogD); u += kThreads) {
-      const int col = ncols + (u >> kLogD), k = u & (D - 1);
-      *reinterpret_cast<__nv_bfloat16*>(Vs + (col >> 6) * (D * 128) + sw128_offset(k, col & 63)) =
-          __float2bfloat16_rn(0.f);
-    }
+    // value rows of this chunk (the same gather as for its codeword rows).  Asynchronous copies: they land
+    // while the chunk's logits are turned into weights.  Padding rows are zero: they meet finite weights.
+    gather_rows(Vs, Vch, e0);
     if (e0 == 0) PHASE_MARK(12);
 
     // ---- child logits: running maximum over non-empty children
@@ -632,7 +618,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const uint32_t aa = smem_u32(CA), va = smem_u32(Vs);
       for (int k = 0; k < np16 / 16; ++k)
         umma_bf16(tmem_base + CT, umma_desc_sw128(aa + (k / 4) * kRows * 128 + (k % 4) * 32),
-                  umma_desc_sw128(va + (k / 4) * D * 128 + (k % 4) * 32), idesc_o, true);
+                  umma_desc_sw128_mn(va + k * 2048, (uint32_t)(np16 * 128)), idesc_o, true);
       umma_commit(bar_pv);
     }
     if (e_next < PC) {
@@ -700,7 +686,7 @@ size_t attend_smem(int D, int CT, int CHW, int NQ) {
 }
 
 template <int D, int NQ, int CT>
-avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUtensorMap& tmVpT,
+avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUtensorMap& tmVpb,
                      const CUtensorMap& tmY, const AttendParams& a, unsigned BH, size_t smem, bool chained,
                      cudaStream_t st) {
   auto kern = tc_attend_kernel<D, NQ, CT>;
@@ -717,15 +703,15 @@ avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUte
   // Inside avq_forward (`chained`) the kernel before it in the stream is the aggregate's finalize kernel
   // and Q was complete before the call, so the attention kernel may start as its programmatic dependent.
   // A stand-alone avq_attend is launched plainly: the work before it in the stream may be producing Q.
-  return cuda_ok(launch_pdl(kern, grid, dim3(128 * NQ), smem, st, chained, tmQ, tmCp, tmVpT, tmY, a));
+  return cuda_ok(launch_pdl(kern, grid, dim3(128 * NQ), smem, st, chained, tmQ, tmCp, tmVpb, tmY, a));
 }
 
 template <int D>
 avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const void* Cc, const float* np_,
-                  const float* nc, const void* VpT, const void* VcT, int32_t P, void* Y, int32_t* topp_out,
+                  const float* nc, const void* Vpb, const void* Vcb, int32_t P, void* Y, int32_t* topp_out,
                   float* importance_out, int32_t* status_word, bool chained, cudaStream_t st) {
   const uint64_t BH = (uint64_t)p.B * p.H;
-  CUtensorMap tmQ, tmCp, tmVpT, tmY;
+  CUtensorMap tmQ, tmCp, tmVpb, tmY;
   {
     const uint64_t dims[3] = {(uint64_t)D, (uint64_t)p.Nq, BH};
     const uint32_t box[3] = {64, (uint32_t)kRows, 1};
@@ -741,14 +727,14 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
     if (s != AVQ_OK) return s;
   }
   {
-    const uint64_t dims[2] = {(uint64_t)p.M, BH * D};
-    const uint32_t box[2] = {64, (uint32_t)D};
-    avq_status s = make_tmap_bf16(&tmVpT, VpT, 2, dims, box);
+    const uint64_t dims[2] = {(uint64_t)D, BH * p.M};
+    const uint32_t box[2] = {64, (uint32_t)p.M};
+    avq_status s = make_tmap_bf16(&tmVpb, Vpb, 2, dims, box);
     if (s != AVQ_OK) return s;
   }
   AttendParams a;
   a.Cc = static_cast<const __nv_bfloat16*>(Cc);
-  a.VcT = static_cast<const __nv_bfloat16*>(VcT);
+  a.Vcb = static_cast<const __nv_bfloat16*>(Vcb);
   a.np_ = np_;
   a.nc = nc;
   a.Y = static_cast<__nv_bfloat16*>(Y);
@@ -770,13 +756,13 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
   // four small CTAs of 128 threads, two of 256, or one of 512.
   const unsigned bh = (unsigned)BH;
   if (D == 64) {
-    if (CT == 64) return launch_nq<D, 1, 64>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
-    if (CT == 128) return launch_nq<D, 2, 128>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
-    return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
+    if (CT == 64) return launch_nq<D, 1, 64>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
+    if (CT == 128) return launch_nq<D, 2, 128>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
+    return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
   }
-  if (CT == 64) return launch_nq<D, 2, 64>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
-  if (CT == 128) return launch_nq<D, 4, 128>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
-  return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpT, tmY, a, bh, smem, chained, st);
+  if (CT == 64) return launch_nq<D, 2, 64>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
+  if (CT == 128) return launch_nq<D, 4, 128>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
+  return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
 }
 
 }  // namespace
@@ -788,10 +774,10 @@ extern "C" __attribute__((visibility("default"))) int avq_debug_phase_clocks(lon
 #endif
 
 avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc, const float* np_,
-                     const float* nc, const void* VpT, const void* VcT, int32_t P, void* Y, int32_t* topp_out,
+                     const float* nc, const void* Vpb, const void* Vcb, int32_t P, void* Y, int32_t* topp_out,
                      float* importance_out, int32_t* status_word, bool chained, cudaStream_t st) {
-  return p.d == 64 ? launch<64>(p, Q, Cp, Cc, np_, nc, VpT, VcT, P, Y, topp_out, importance_out, status_word, chained, st)
-                   : launch<128>(p, Q, Cp, Cc, np_, nc, VpT, VcT, P, Y, topp_out, importance_out, status_word, chained, st);
+  return p.d == 64 ? launch<64>(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, P, Y, topp_out, importance_out, status_word, chained, st)
+                   : launch<128>(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, P, Y, topp_out, importance_out, status_word, chained, st);
 }
 
 }  // namespace avq

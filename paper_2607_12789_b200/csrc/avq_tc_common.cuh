@@ -219,6 +219,19 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t addr) {
   d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
   return d;
 }
+// Shared-memory descriptor of an MN-major operand: row k of the tile holds 64 consecutive M/N elements
+// (128 bytes, 128-byte swizzle), 8-row groups 1024 bytes apart along K, further 64-element groups along
+// M/N `group_bytes` apart.  `addr` is the address of the first row of the K step (16 rows = 2048 bytes per
+// step).  The instruction descriptor must mark the operand MN-major (bit 16 for B).
+__device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t addr, uint32_t group_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((group_bytes >> 4) & 0x3FFFu) << 16;   // leading byte offset: next 64-element group
+  d |= (uint64_t)(1024 >> 4) << 32;                      // stride byte offset: next 8-row group along K
+  d |= (uint64_t)1 << 46;                                // descriptor version for sm_100
+  d |= (uint64_t)2 << 61;                                // SWIZZLE_128B
+  return d;
+}
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                           bool accumulate) {
   asm volatile(
