@@ -43,8 +43,8 @@ METRIC = "avq_attn_fwd_query_tokens_per_s"
 # summarised under profiles/ (tc_attend_c1.md, tc_attend_c3.md, tc_assign_c3.md); other workloads: None.
 NCU_TRAFFIC = {
     ("c1_vitb", "assign"): 13.12e6, ("c1_vitb", "aggregate"): 17.67e6 + 6.40e6, ("c1_vitb", "attend"): 14.79e6,
-    ("c3_long", "assign"): 71.58e6 + 2.33e6, ("c3_long", "aggregate"): 75.16e6 + 0.86e6 + 8.46e6,
-    ("c3_long", "attend"): 71.51e6 + 28.73e6,
+    ("c3_long", "assign"): 71.58e6 + 2.68e6, ("c3_long", "aggregate"): 75.16e6 + 0.92e6 + 8.46e6,
+    ("c3_long", "attend"): 71.51e6 + 28.71e6,
 }
 UNIT = "query-tokens/s"
 
