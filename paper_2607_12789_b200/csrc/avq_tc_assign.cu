@@ -21,8 +21,8 @@ using namespace tc;
 constexpr int kKeys = 128;
 constexpr int kThreadsA = 256;
 // CTAs per SM the register budget is set for: the d = 64 kernels are small enough (24-48 KB of shared
-// memory, at most 128 TMEM columns up to M = 128) for four (C = 4) or three (C = 8) to share an SM.
-constexpr int assign_min_ctas(int D, int NL) { return D == 64 ? (NL == 1 ? 4 : 3) : 2; }
+// memory, at most 128 TMEM columns up to M = 128) for four to share an SM.
+constexpr int assign_min_ctas(int D, int NL) { return D == 64 ? 4 : 2; }
 
 #ifdef AVQ_PHASE_DEBUG
 __device__ long long g_assign_clocks[64 * 16];
