@@ -45,6 +45,7 @@ struct AttendParams {
   float* importance_out;      // optional
   int32_t* status_word;
   int H, Nq, M, C, P, nblk;
+  int total_tiles;            // nblk * B * H
   int logC;                   // log2(C)
   uint32_t tmem_cols;
   float scale_log2e;
@@ -156,20 +157,42 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   float* xz2 = xz + NQ * kRows;                          // [NQ][128]
   int* sel_list = reinterpret_cast<int*>(xz2 + NQ * kRows);   // [256]
   uint32_t* wmask = reinterpret_cast<uint32_t*>(sel_list + 256);   // [16]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(wmask + 18);        // [4]  (wmask[16] is a scratch word)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(wmask + 18);        // [5]  (wmask[16] is a scratch word)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int q = warp & 3, cq = warp >> 2, r = q * 32 + lane;
-  const int blk = blockIdx.x, bh = blockIdx.y, h = bh % p.H;
-  const int i0 = blk * kRows;
-  const int rows_valid = min(kRows, p.Nq - i0);
   const int colbase = cq * QW;
-  uint64_t* bar_ld0 = &bars[0];
-  uint64_t* bar_ld1 = &bars[1];
+  uint64_t* bar_q = &bars[0];                            // query tile landed
+  uint64_t* bar_ld1 = &bars[1];                          // parent value rows landed
   uint64_t* bar_s = &bars[2];
   uint64_t* bar_pv = &bars[3];
+  uint64_t* bar_cp = &bars[4];                           // parent codebook landed
+  // A CTA works through the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  With one tile per CTA (the small
+  // shapes, several CTAs per SM) the loop runs once.  The large shapes (CT >= 128: one or two CTAs per SM)
+  // launch one wave of CTAs; the next tile's Q is loaded as soon as this tile's last logits are done, its
+  // codebook and value rows as soon as this tile's last value MMA is done, so the set-up, the loads and the
+  // first MMA of a tile hide behind the tail of the tile before.
+  constexpr bool kChain = CT >= 128;                     // the output is staged in CC, Qs is free for the next Q
+  auto issue_q = [&](int t) {                            // thread 0 only
+    const int tb = t / p.nblk, ti0 = (t - tb * p.nblk) * kRows;
+    mbar_expect_tx(bar_q, (uint32_t)(kSubD * kRows * 128));
+#pragma unroll
+    for (int s = 0; s < kSubD; ++s) tma_load_3d(Qs + s * kRows * 128, &tmQ, s * 64, ti0, tb, bar_q);
+  };
+  auto issue_cp = [&](int t) {
+    const int th = (t / p.nblk) % p.H;
+    mbar_expect_tx(bar_cp, (uint32_t)(kSubD * M * 128));
+#pragma unroll
+    for (int s = 0; s < kSubD; ++s) tma_load_2d(CA + s * M * 128, &tmCp, s * 64, th * M, bar_cp);
+  };
+  auto issue_vp = [&](int t) {
+    const int tb = t / p.nblk;
+    mbar_expect_tx(bar_ld1, (uint32_t)(kSubD * M * 128));
+#pragma unroll
+    for (int s = 0; s < kSubD; ++s) tma_load_2d(Vs + s * M * 128, &tmVpb, s * 64, tb * M, bar_ld1);
+  };
 
   __shared__ int early_exit;
   PHASE_MARK(0);
@@ -181,18 +204,15 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmCp);
     prefetch_tmap(&tmVpb);
-    mbar_init(bar_ld0, 1);
+    mbar_init(bar_q, 1);
+    mbar_init(bar_cp, 1);
     mbar_init(bar_ld1, 1);
     mbar_init(bar_s, 1);
     mbar_init(bar_pv, 1);
     mbar_fence_init();
     *abort_flag = 0;
-    mbar_expect_tx(bar_ld0, (uint32_t)(kSubD * (kRows + M) * 128));
-#pragma unroll
-    for (int s = 0; s < kSubD; ++s) {
-      tma_load_3d(Qs + s * kRows * 128, &tmQ, s * 64, i0, bh, bar_ld0);
-      tma_load_2d(CA + s * M * 128, &tmCp, s * 64, h * M, bar_ld0);
-    }
+    issue_q(blockIdx.x);
+    issue_cp(blockIdx.x);
   }
   if (warp == 1) {                                   // not the warp whose lane 0 is busy issuing the loads
     tmem_alloc(tmem_slot, p.tmem_cols);
@@ -209,8 +229,21 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const uint32_t idesc_o = umma_idesc_bf16(kRows, D) | (1u << 16);   // B (the value rows) is MN-major
   const float sc = p.scale_log2e;
   PHASE_MARK(1);
+  uint32_t ph_s = 0, ph_pv = 0, ph_in = 0;               // ph_in: parity of the three load barriers (once per tile)
+  const int PC = P * C;
+  const int my_cols = min(max(M - colbase, 0), QW);      // multiple of 16 (M % 32 == 0, QW % 16 == 0)
+  bool first = true;
+  for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+  const int bh = tile / p.nblk, blk = tile - bh * p.nblk, h = bh % p.H;
+  const int i0 = blk * kRows;
+  const int rows_valid = min(kRows, p.Nq - i0);
+  const int next_tile = tile + gridDim.x;
+  const bool has_next = kChain && next_tile < p.total_tiles;
   if (tid == 0) {
-    if (mbar_wait(bar_ld0, 0, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND)) {
+    if (!first) tma_store_wait_read();                   // the output tile of the tile before has left CC
+    const bool q_ok = mbar_wait(bar_q, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+    const bool c_ok = mbar_wait(bar_cp, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+    if (q_ok && c_ok) {
       tc_fence_after();
       const uint32_t idesc = umma_idesc_bf16(kRows, M);
       const uint32_t qa = smem_u32(Qs), ca = smem_u32(CA);
@@ -223,13 +256,13 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   }
 
   // ---- Part 2 reads what the earlier kernels of this call wrote: status word, counts, value sums.
-  pdl_wait();
-  if (tid == 0) {
-    // a wait that expired in an earlier CTA or kernel of this call: do not start more work
-    early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
-    mbar_expect_tx(bar_ld1, (uint32_t)(kSubD * M * 128));
-#pragma unroll
-    for (int s = 0; s < kSubD; ++s) tma_load_2d(Vs + s * M * 128, &tmVpb, s * 64, bh * M, bar_ld1);
+  if (first) {
+    pdl_wait();
+    if (tid == 0) {
+      // a wait that expired in an earlier CTA or kernel of this call: do not start more work
+      early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
+      issue_vp(tile);
+    }
   }
   for (int j = tid; j < CT; j += kThreads) {
     const float n = j < M ? p.np_[(size_t)bh * M + j] : 0.f;
@@ -238,7 +271,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     cntk[j] = n;
   }
   __syncthreads();
-  if (early_exit) {
+  if (first && early_exit) {
     // let the MMA and the load already in flight finish, then leave cleanly
     mbar_wait(bar_s, 0, abort_flag, nullptr, 0);
     mbar_wait(bar_ld1, 0, abort_flag, nullptr, 0);
@@ -247,15 +280,14 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
     return;
   }
-  uint32_t ph_s = 0, ph_pv = 0;
-  const int PC = P * C;
-  const int my_cols = min(max(M - colbase, 0), QW);      // multiple of 16 (M % 32 == 0, QW % 16 == 0)
+  first = false;
 
   // ---- parents: row maximum over non-empty codewords (empty ones carry a -inf bias)
   PHASE_MARK(2);
   mbar_wait(bar_s, ph_s, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
   ph_s ^= 1;
   tc_fence_after();
+  if (tid == 0 && has_next && PC == 0) issue_q(next_tile);   // no child logits will read this Q tile
   PHASE_MARK(3);
   // This thread's QW (<= 64) parent logits are read from TMEM once and stay in registers through the
   // maximum, the exponentials, the importance sums and the conversion to bf16.
@@ -480,7 +512,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // ---- bf16 weights into shared memory (over the dead codebook) + their denominator.  A refined parent
   // is removed from the numerator by clearing its row of the value tile (d / 8 16-byte stores) and from the
   // denominator by its zeroed count, so the weights themselves need no mask.
-  mbar_wait(bar_ld1, 0, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);   // value sums have landed
+  mbar_wait(bar_ld1, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);   // value sums have landed
   for (int u = tid; u < (min(P, M) << kLogChunks); u += kThreads) {
     const int row = sel_list[u >> kLogChunks], ch = u & ((1 << kLogChunks) - 1);
     *reinterpret_cast<uint4*>(Vs + (ch >> 3) * (M * 128) + sw128_offset(row, (ch & 7) * 8)) = make_uint4(0, 0, 0, 0);
@@ -510,7 +542,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // ---- O = A . Vbar_p, and right behind it the first child chunk's logits
   if (tid == 0) {
     tc_fence_after();
-    if (mbar_wait(bar_ld1, 0, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND)) {
+    if (mbar_wait(bar_ld1, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND)) {
       const uint32_t aa = smem_u32(CA), va = smem_u32(Vs);
       for (int k = 0; k < M / 16; ++k)
         umma_bf16(tmem_base + CT, umma_desc_sw128(aa + (k / 4) * kRows * 128 + (k % 4) * 32),
@@ -549,6 +581,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     mbar_wait(bar_s, ph_s, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
     ph_s ^= 1;
     tc_fence_after();
+    if (tid == 0 && has_next && e0 + CHW >= PC) issue_q(next_tile);   // the last logits are done: Q is dead
     if (e0 == 0) PHASE_MARK(13);
     const int my_c = min(max(np16 - cq * QWC, 0), QWC);
     float mxc = -INFINITY;
@@ -645,11 +678,20 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // ---- epilogue: Y = O / z
   PHASE_MARK(26);
   const bool o_ok = mbar_wait(bar_pv, ph_pv, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+  ph_pv ^= 1;
   tc_fence_after();
+  // the last value MMA has released the weight tile and the value tile: the next tile's codebook and
+  // parent value rows load while this tile's output is written
+  if (tid == 0 && has_next) {
+    issue_cp(next_tile);
+    issue_vp(next_tile);
+  }
   PHASE_MARK(27);
+  // The output tile is staged in shared memory in the layout of the Q load and written with TMA tile
+  // stores; rows past Nq are clipped by the tensor map.  Staging area: the child-code buffer where it is as
+  // large as a Q tile (its codes are consumed), else the Q tile, which no MMA reads any more.
+  unsigned char* stage = kChain ? CC : Qs;
   if (o_ok) {
-    // The output tile is staged in shared memory (over the Q tile, which no MMA reads any more) in the
-    // layout of the Q load and written with TMA tile stores; rows past Nq are clipped by the tensor map.
     const float inv = 1.f / z_run;
     for (int c0 = 0; c0 < D / NQ; c0 += 16) {
       float o[16];
@@ -658,7 +700,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
       for (int e = 0; e < 16; e += 2) pk[e >> 1] = pack_bf16(o[e] * inv, o[e + 1] * inv);
       const int col0 = cq * (D / NQ) + c0;
-      unsigned char* sub = Qs + (col0 >> 6) * (kRows * 128);
+      unsigned char* sub = stage + (col0 >> 6) * (kRows * 128);
       *reinterpret_cast<uint4*>(sub + sw128_offset(r, col0 & 63)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       *reinterpret_cast<uint4*>(sub + sw128_offset(r, (col0 & 63) + 8)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
     }
@@ -668,9 +710,12 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   __syncthreads();
   if (tid == 0 && o_ok) {
 #pragma unroll
-    for (int s2 = 0; s2 < kSubD; ++s2) tma_store_3d(&tmY, Qs + s2 * kRows * 128, s2 * 64, i0, bh);
-    tma_store_commit_and_wait_read();
+    for (int s2 = 0; s2 < kSubD; ++s2) tma_store_3d(&tmY, stage + s2 * kRows * 128, s2 * 64, i0, bh);
+    tma_store_commit();
+    if (!has_next) tma_store_wait_read();              // before the CTA may leave (or: waited at the next tile)
   }
+  ph_in ^= 1;
+  }   // tiles
   PHASE_MARK(28);
   if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
   PHASE_MARK(29);
@@ -681,7 +726,7 @@ size_t attend_smem(int D, int CT, int CHW, int NQ) {
   const size_t ca = (size_t)max(CT * D * 2, subA * kRows * 128);
   size_t b = (size_t)(D / 64) * kRows * 128 + ca + (size_t)subA * D * 128 + (size_t)CHW * D * 2;
   b += sizeof(float) * (3 * (size_t)CT + 2 * (size_t)CHW + 256 + 4 * (size_t)CT + 3 * (size_t)NQ * kRows);
-  b += sizeof(int) * 256 + sizeof(uint32_t) * 18 + sizeof(uint64_t) * 4 + 2 * sizeof(uint32_t);
+  b += sizeof(int) * 256 + sizeof(uint32_t) * 18 + sizeof(uint64_t) * 5 + 2 * sizeof(uint32_t);
   return b + 64;
 }
 
@@ -699,7 +744,17 @@ avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUte
       return AVQ_ERR_CUDA;
     if (dev >= 0 && dev < 64) configured[dev] = smem;
   }
-  dim3 grid(a.nblk, BH);
+  // Grid: one CTA per tile for the small shapes; one wave of CTAs, each taking every gridDim.x-th tile, for
+  // the shapes whose CTAs chain their tiles (CT >= 128: 4 / NQ CTAs per SM).
+  static int sm_count[64] = {};
+  int sms = (dev >= 0 && dev < 64) ? sm_count[dev] : 0;
+  if (sms <= 0) {
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return AVQ_ERR_CUDA;
+    if (dev >= 0 && dev < 64) sm_count[dev] = sms;
+  }
+  int ctas = a.total_tiles;
+  if (CT >= 128 && ctas > (4 / NQ) * sms) ctas = (4 / NQ) * sms;
+  const dim3 grid((unsigned)ctas);
   // Inside avq_forward (`chained`) the kernel before it in the stream is the aggregate's finalize kernel
   // and Q was complete before the call, so the attention kernel may start as its programmatic dependent.
   // A stand-alone avq_attend is launched plainly: the work before it in the stream may be producing Q.
@@ -743,6 +798,8 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
   a.status_word = status_word;
   a.H = p.H; a.Nq = p.Nq; a.M = p.M; a.C = p.C; a.P = P;
   a.nblk = (p.Nq + kRows - 1) / kRows;
+  if ((uint64_t)a.nblk * BH > 0x7fffffffull) return AVQ_ERR_UNSUPPORTED;
+  a.total_tiles = (int)(a.nblk * BH);
   const int CT = p.M <= 64 ? 64 : (p.M <= 128 ? 128 : 256);
   const int CHW = CT < 128 ? CT : 128;
   a.logC = p.C == 8 ? 3 : 2;
