@@ -233,6 +233,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int PC = P * C;
   const int my_cols = min(max(M - colbase, 0), QW);      // multiple of 16 (M % 32 == 0, QW % 16 == 0)
   bool first = true;
+  bool store_pending = false;                            // thread 0: a TMA store may still be reading CC
   for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
   const int bh = tile / p.nblk, blk = tile - bh * p.nblk, h = bh % p.H;
   const int i0 = blk * kRows;
@@ -240,7 +241,6 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int next_tile = tile + gridDim.x;
   const bool has_next = kChain && next_tile < p.total_tiles;
   if (tid == 0) {
-    if (!first) tma_store_wait_read();                   // the output tile of the tile before has left CC
     const bool q_ok = mbar_wait(bar_q, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
     const bool c_ok = mbar_wait(bar_cp, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
     if (q_ok && c_ok) {
@@ -465,6 +465,12 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       cntk[j] = 0.f;
       if (p.topp_out) p.topp_out[((size_t)bh * p.nblk + blk) * P + pos] = j;
     }
+  }
+  // the output tile of the tile before must have left the child-code buffer before it is refilled (its
+  // store was issued a whole parent pass ago, so this does not wait in practice)
+  if (tid == 0 && store_pending) {
+    tma_store_wait_read();
+    store_pending = false;
   }
   __syncthreads();
   PHASE_MARK(8);
@@ -712,7 +718,8 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
     for (int s2 = 0; s2 < kSubD; ++s2) tma_store_3d(&tmY, stage + s2 * kRows * 128, s2 * 64, i0, bh);
     tma_store_commit();
-    if (!has_next) tma_store_wait_read();              // before the CTA may leave (or: waited at the next tile)
+    if (has_next) store_pending = true;                // waited for before the next tile refills CC
+    else tma_store_wait_read();                        // before the CTA may leave
   }
   ph_in ^= 1;
   }   // tiles
