@@ -169,12 +169,15 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   uint64_t* bar_s = &bars[2];
   uint64_t* bar_pv = &bars[3];
   uint64_t* bar_cp = &bars[4];                           // parent codebook landed
-  // A CTA works through the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  With one tile per CTA (the small
-  // shapes, several CTAs per SM) the loop runs once.  The large shapes (CT >= 128: one or two CTAs per SM)
-  // launch one wave of CTAs; the next tile's Q is loaded as soon as this tile's last logits are done, its
-  // codebook and value rows as soon as this tile's last value MMA is done, so the set-up, the loads and the
-  // first MMA of a tile hide behind the tail of the tile before.
-  constexpr bool kChain = CT >= 128;                     // the output is staged in CC, Qs is free for the next Q
+  // A CTA works through the tiles blockIdx.x, blockIdx.x + gridDim.x, ... (the grid is one wave of CTAs).
+  // The next tile's Q is loaded as soon as this tile's last logits are done, its codebook as soon as this
+  // tile's last value MMA is done, so the set-up, the loads and the first MMA of a tile hide behind the tail
+  // of the tile before.  The output is staged where the next tile's first loads do not go: in the child-code
+  // buffer when that is as large as a Q tile (CT >= 128), else across the value tile and the child-code
+  // buffer, which are adjacent and together as large (the next tile's value rows then load a little later).
+  constexpr bool kChain = true;
+  constexpr bool kStageInCC = CT >= 128;
+  static_assert(kStageInCC || (CT * D * 2 + CHW * D * 2 == kSubD * kRows * 128), "staging area");
   auto issue_q = [&](int t) {                            // thread 0 only
     const int tb = t / p.nblk, ti0 = (t - tb * p.nblk) * kRows;
     mbar_expect_tx(bar_q, (uint32_t)(kSubD * kRows * 128));
@@ -253,6 +256,12 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                   umma_desc_sw128(ca + (k / 4) * M * 128 + (k % 4) * 32), idesc, k > 0);
     }
     umma_commit(bar_s);
+    if (!kStageInCC && !first) {
+      // the value tile was the staging area of the tile before: reload it once that store has read it
+      tma_store_wait_read();
+      store_pending = false;
+      issue_vp(tile);
+    }
   }
 
   // ---- Part 2 reads what the earlier kernels of this call wrote: status word, counts, value sums.
@@ -690,13 +699,12 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // parent value rows load while this tile's output is written
   if (tid == 0 && has_next) {
     issue_cp(next_tile);
-    issue_vp(next_tile);
+    if (kStageInCC) issue_vp(next_tile);
   }
   PHASE_MARK(27);
   // The output tile is staged in shared memory in the layout of the Q load and written with TMA tile
-  // stores; rows past Nq are clipped by the tensor map.  Staging area: the child-code buffer where it is as
-  // large as a Q tile (its codes are consumed), else the Q tile, which no MMA reads any more.
-  unsigned char* stage = kChain ? CC : Qs;
+  // stores; rows past Nq are clipped by the tensor map.  Staging area: see the top of the tile loop.
+  unsigned char* stage = kStageInCC ? CC : Vs;
   if (o_ok) {
     const float inv = 1.f / z_run;
     for (int c0 = 0; c0 < D / NQ; c0 += 16) {
@@ -751,8 +759,7 @@ avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUte
       return AVQ_ERR_CUDA;
     if (dev >= 0 && dev < 64) configured[dev] = smem;
   }
-  // Grid: one CTA per tile for the small shapes; one wave of CTAs, each taking every gridDim.x-th tile, for
-  // the shapes whose CTAs chain their tiles (CT >= 128: 4 / NQ CTAs per SM).
+  // Grid: one wave of CTAs (4 / NQ per SM), each taking every gridDim.x-th tile.
   static int sm_count[64] = {};
   int sms = (dev >= 0 && dev < 64) ? sm_count[dev] : 0;
   if (sms <= 0) {
@@ -760,7 +767,7 @@ avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUte
     if (dev >= 0 && dev < 64) sm_count[dev] = sms;
   }
   int ctas = a.total_tiles;
-  if (CT >= 128 && ctas > (4 / NQ) * sms) ctas = (4 / NQ) * sms;
+  if (ctas > (4 / NQ) * sms) ctas = (4 / NQ) * sms;
   const dim3 grid((unsigned)ctas);
   // Inside avq_forward (`chained`) the kernel before it in the stream is the aggregate's finalize kernel
   // and Q was complete before the call, so the attention kernel may start as its programmatic dependent.
