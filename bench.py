@@ -43,10 +43,10 @@ METRIC = "avq_attn_fwd_query_tokens_per_s"
 # summarised under profiles/ (tc_attend_c1.md, tc_attend_c3.md, tc_assign_c3.md, kernels_c2_and_N16384_M64_P8.md);
 # other workloads: None.
 NCU_TRAFFIC = {
-    ("c1_vitb", "assign"): 13.12e6, ("c1_vitb", "aggregate"): 17.67e6 + 6.40e6, ("c1_vitb", "attend"): 14.79e6,
+    ("c1_vitb", "assign"): 13.12e6, ("c1_vitb", "aggregate"): 17.67e6 + 6.40e6, ("c1_vitb", "attend"): 14.80e6,
     ("c2_mid", "assign"): 19.06e6, ("c2_mid", "aggregate"): 22.55e6 + 8.54e6, ("c2_mid", "attend"): 19.19e6,
     ("c3_long", "assign"): 71.58e6 + 2.68e6, ("c3_long", "aggregate"): 75.16e6 + 0.92e6 + 8.46e6,
-    ("c3_long", "attend"): 71.51e6 + 24.34e6,
+    ("c3_long", "attend"): 71.52e6 + 25.32e6,
 }
 UNIT = "query-tokens/s"
 
