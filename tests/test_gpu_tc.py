@@ -157,3 +157,10 @@ def test_single_query_block_shorter_than_a_tile_and_tiny_key_set():
     x = synth.generate(wl)
     x["Q"] = np.ascontiguousarray(x["Q"][:, :, :1])
     parity.full_parity(wl, x=x)
+
+
+def test_chained_tiles_with_several_child_chunks():
+    """More tiles than one wave of CTAs (every CTA takes several tiles in a row) with every parent refined, so
+    that each tile runs through several child chunks before the next tile's loads are issued."""
+    parity.sampled_parity(synth.sweep_point(16384, 64, 64), heads=[(0, 7)], blocks_per_head=4)
+    parity.sampled_parity(synth.sweep_point(16384, 256, 64).with_(H=4), heads=[(0, 2)], blocks_per_head=3)
