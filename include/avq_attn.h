@@ -69,7 +69,8 @@ typedef enum {
   AVQ_ERR_ALIGN = 4,          /* a pointer is not 16-byte aligned                          */
   AVQ_ERR_WORKSPACE = 5,      /* workspace missing or smaller than avq_workspace_bytes()  */
   AVQ_ERR_CUDA = 6,           /* a CUDA runtime / driver call failed                      */
-  AVQ_ERR_DEVICE_TIMEOUT = 7  /* a bounded device-side wait expired (see avq_check)       */
+  AVQ_ERR_DEVICE_TIMEOUT = 7, /* a bounded device-side wait expired (see avq_check)       */
+  AVQ_ERR_INDEX = 8           /* a kernel met a parent/child index out of range (avq_check) */
 } avq_status;
 
 typedef enum { AVQ_F32 = 0, AVQ_BF16 = 1 } avq_dtype;
@@ -98,7 +99,9 @@ typedef struct {
 
 /* Supported envelope.
  *   CUDA-core kernels (float32, or AVQ_FLAG_SIMT): d % 4 == 0, 4 <= d <= 256; 1 <= M <= 1024;
- *     1 <= C <= 16; 0 <= P <= M; 1 <= block_q <= 256; M + P*C <= 8192.
+ *     1 <= C <= 16; 0 <= P <= M; 1 <= block_q <= 256; M + P*C <= 8192; and the attention kernel's
+ *     shared memory, 4*block_q*(d + 2) + 20*M + 32*(M + P*C) + 4*max(P, 1) bytes, at most 200 KiB
+ *     (e.g. d = 256 with block_q = 256 does not fit; d = 128 with block_q = 256 does).
  *   Tensor-core kernels (bfloat16, no flags): d in {64, 128}; M a multiple of 32, 32..256;
  *     C in {4, 8}; 0 <= P <= M; block_q = 128; scale > 0; AVQ_FLAG_PARENT_STAYS clear.
  */
@@ -121,7 +124,9 @@ AVQ_API avq_status avq_assign(const avq_problem* prob, const void* K, const void
  * Vc[b,h,m,c,:], nc[b,h,m,c] the same over keys with (parent, child) = (m, c); keys with
  * child index -1 enter the parent sums only.  All four outputs are float32 and are
  * overwritten (the call zeroes them first).  Summation order is not fixed, so the last
- * bits of the sums may differ from run to run; counts are exact. */
+ * bits of the sums may differ from run to run; counts are exact.
+ * Indices are the caller's here: a key whose parent index is outside [0, M) or whose child
+ * index is outside [-1, C) is left out of every sum (no out-of-range access is made). */
 AVQ_API avq_status avq_aggregate(const avq_problem* prob, const void* V, const int32_t* parent_idx,
                          const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc,
                          void* stream);
@@ -204,7 +209,8 @@ AVQ_API avq_status avq_workspace_layout(const avq_problem* prob, int32_t P, int3
 
 /* Waits for `stream`, reads the status word in the workspace header and clears it.
  * AVQ_OK, AVQ_ERR_DEVICE_TIMEOUT (a bounded wait inside a kernel expired; outputs of that
- * call are not valid) or AVQ_ERR_CUDA.  Blocks the host. */
+ * call are not valid), AVQ_ERR_INDEX (a kernel skipped a key whose index was out of range)
+ * or AVQ_ERR_CUDA.  Blocks the host. */
 AVQ_API avq_status avq_check(void* workspace, void* stream);
 
 /* Static, NUL-terminated description of a status code. */

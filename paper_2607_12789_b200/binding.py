@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "lib", "libavq_attn.so")
 AVQ_F32, AVQ_BF16 = 0, 1
 FLAG_PARENT_STAYS, FLAG_SIMT = 1, 2
 STATUS_NAMES = {0: "AVQ_OK", 1: "AVQ_ERR_NULL", 2: "AVQ_ERR_SHAPE", 3: "AVQ_ERR_UNSUPPORTED", 4: "AVQ_ERR_ALIGN",
-                5: "AVQ_ERR_WORKSPACE", 6: "AVQ_ERR_CUDA", 7: "AVQ_ERR_DEVICE_TIMEOUT"}
+                5: "AVQ_ERR_WORKSPACE", 6: "AVQ_ERR_CUDA", 7: "AVQ_ERR_DEVICE_TIMEOUT", 8: "AVQ_ERR_INDEX"}
 
 EXPORTS = ("avq_workspace_bytes", "avq_assign", "avq_aggregate", "avq_forward", "avq_forward_host", "avq_attend",
            "avq_workspace_layout", "avq_check", "avq_status_string", "avq_version", "avq_forward_static",

@@ -23,7 +23,7 @@ NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
     "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-] + os.environ.get("AVQ_NVCC_EXTRA", "").split()
+]
 
 
 def _nvcc() -> str:
@@ -31,6 +31,19 @@ def _nvcc() -> str:
     if not os.path.exists(exe):
         raise RuntimeError("nvcc not found; the CUDA extension cannot be built")
     return exe
+
+
+def source_hash() -> str:
+    """Short digest of every kernel source and header the library is built from: identifies which
+    sources a profiler capture (or any other stored measurement) belongs to."""
+    import hashlib
+    h = hashlib.sha256()
+    files = [os.path.join(ROOT, "include", "avq_attn.h")]
+    files += sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh", ".h")))
+    for path in files:
+        h.update(os.path.basename(path).encode())
+        h.update(open(path, "rb").read())
+    return h.hexdigest()[:16]
 
 
 def _newest_header() -> float:

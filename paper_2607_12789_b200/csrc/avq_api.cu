@@ -48,6 +48,7 @@ avq_status validate_forward(const avq_problem* p, int32_t P, int32_t block_q) {
   } else {
     if (block_q > 256) return AVQ_ERR_UNSUPPORTED;
     if ((int64_t)p->M + (int64_t)P * p->C > 8192) return AVQ_ERR_UNSUPPORTED;
+    if (simt_attend_smem_bytes(p->d, p->M, p->C, P, block_q) > kSimtAttendSmemLimit) return AVQ_ERR_UNSUPPORTED;
   }
   return AVQ_OK;
 }
@@ -60,11 +61,11 @@ Layout make_layout(const avq_problem& p, int32_t /*P*/, int32_t /*block_q*/) {
   L.header = 0;
   L.Vc = take(sizeof(float) * BH * p.M * p.C * p.d);
   L.nc = take(sizeof(float) * BH * p.M * p.C);
+  L.Vp = take(sizeof(float) * BH * p.M * p.d);
+  L.np = take(sizeof(float) * BH * p.M);
   L.zero_end = off;
   L.parent_idx = take(sizeof(int32_t) * BH * p.Nk);
   L.child_idx = take(sizeof(int32_t) * BH * p.Nk);
-  L.Vp = take(sizeof(float) * BH * p.M * p.d);
-  L.np = take(sizeof(float) * BH * p.M);
   if (use_tensor_path(p)) {
     L.Vpb = take(2 * BH * p.M * p.d);
     L.Vcb = take(2 * BH * p.M * p.C * p.d);
@@ -122,7 +123,7 @@ avq_status avq_aggregate(const avq_problem* prob, const void* V, const int32_t* 
     return AVQ_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (use_tensor_path(*prob))
-    return tc_aggregate(*prob, V, parent_idx, child_idx, Vp, np_, Vc, nc, nullptr, nullptr, false, st);
+    return tc_aggregate(*prob, V, parent_idx, child_idx, Vp, np_, Vc, nc, nullptr, nullptr, false, nullptr, st);
   return simt_aggregate(*prob, V, parent_idx, child_idx, Vp, np_, Vc, nc, st);
 }
 
@@ -184,7 +185,7 @@ avq_status avq_forward(const avq_problem* prob, const void* Q, const void* K, co
     // status header, leaf sums and leaf counts are adjacent: the assign grid clears them on the side
     s = tc_assign(p, K, Cp, Cc, r.pidx, r.cidx, r.status_word, workspace, L.zero_end, st);
     if (s != AVQ_OK) return s;
-    s = tc_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, r.Vpb, r.Vcb, true, st);
+    s = tc_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, r.Vpb, r.Vcb, true, r.status_word, st);
   } else {
     if (cudaMemsetAsync(r.status_word, 0, 256, st) != cudaSuccess) return AVQ_ERR_CUDA;
     s = simt_assign(p, K, Cp, Cc, r.pidx, r.cidx, st);
@@ -243,7 +244,7 @@ avq_status avq_check(void* workspace, void* stream) {
   if (word != 0) {
     if (cudaMemsetAsync(workspace, 0, sizeof(word), st) != cudaSuccess) return AVQ_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return AVQ_ERR_CUDA;
-    return AVQ_ERR_DEVICE_TIMEOUT;
+    return word == DEV_BAD_INDEX ? AVQ_ERR_INDEX : AVQ_ERR_DEVICE_TIMEOUT;
   }
   return AVQ_OK;
 }
@@ -258,6 +259,7 @@ const char* avq_status_string(avq_status s) {
     case AVQ_ERR_WORKSPACE: return "workspace is NULL or too small";
     case AVQ_ERR_CUDA: return "a CUDA call failed";
     case AVQ_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case AVQ_ERR_INDEX: return "a parent or child index read by a kernel was out of range";
   }
   return "unknown status";
 }

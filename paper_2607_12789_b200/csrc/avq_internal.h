@@ -12,13 +12,13 @@ namespace avq {
 // Byte offsets of the regions of an avq_forward workspace.
 struct Layout {
   size_t header = 0;       // 256 bytes; int32 status word at offset 0
-  size_t Vc = 0;           // f32 [B,H,M,C,d]   header, Vc and nc are adjacent: one memset clears them
+  size_t Vc = 0;           // f32 [B,H,M,C,d]   header, Vc, nc, Vp and np are adjacent: one pass clears them
   size_t nc = 0;           // f32 [B,H,M,C]
+  size_t Vp = 0;           // f32 [B,H,M,d]     (accumulates the keys that stay with their parent)
+  size_t np = 0;           // f32 [B,H,M]
   size_t zero_end = 0;     // end of the region that must be zero before aggregation
   size_t parent_idx = 0;   // int32 [B,H,Nk]
   size_t child_idx = 0;    // int32 [B,H,Nk]
-  size_t Vp = 0;           // f32 [B,H,M,d]
-  size_t np = 0;           // f32 [B,H,M]
   size_t Vpb = 0;          // bf16 [B,H,M,d]      copy of Vp (tensor-core path only)
   size_t Vcb = 0;          // bf16 [B,H,M,C,d]    copy of Vc (tensor-core path only)
   size_t total = 0;
@@ -29,6 +29,8 @@ enum DeviceCode : int32_t {
   DEV_OK = 0,
   DEV_TIMEOUT_ASSIGN = 101,
   DEV_TIMEOUT_ATTEND = 102,
+  DEV_TIMEOUT_TEST = 103,      // the self-test wait of avq_selftest_wait_expiry
+  DEV_BAD_INDEX = 201,         // a caller-supplied parent / child index was out of range (the key was skipped)
 };
 
 bool use_tensor_path(const avq_problem& p);
@@ -47,6 +49,10 @@ avq_status simt_attend(const avq_problem& p, const void* Q, const void* Cp, cons
                        int32_t block_q, void* Y, int32_t* topp_out, float* importance_out,
                        cudaStream_t st);
 
+// Shared memory the CUDA-core attention kernel needs for a problem, and the most it may ask for.
+size_t simt_attend_smem_bytes(int d, int M, int C, int P, int block_q);
+constexpr size_t kSimtAttendSmemLimit = 200 * 1024;
+
 // ---- tensor-core kernels (avq_tc_*.cu) ----
 // zero_base / zero_bytes: a region (multiple of 16 bytes, or none) the assign grid clears on the side
 avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const void* Cc,
@@ -54,7 +60,7 @@ avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const 
                      size_t zero_bytes, cudaStream_t st);
 avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
                         const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc,
-                        void* Vpb, void* Vcb, bool pre_zeroed, cudaStream_t st);
+                        void* Vpb, void* Vcb, bool pre_zeroed, int32_t* status_word, cudaStream_t st);
 avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc,
                      const float* np_, const float* nc, const void* Vpb, const void* Vcb, int32_t P,
                      void* Y, int32_t* topp_out, float* importance_out, int32_t* status_word,

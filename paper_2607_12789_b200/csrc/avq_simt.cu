@@ -353,7 +353,9 @@ __global__ void __launch_bounds__(kAttendThreads) attend_simt_kernel(AttendArgs 
   }
 }
 
-size_t attend_smem_bytes(int d, int M, int C, int P, int block_q) {
+}  // namespace (the size below is also used by the host-side validation)
+
+size_t simt_attend_smem_bytes(int d, int M, int C, int P, int block_q) {
   const size_t ncols = (size_t)M + (size_t)P * C;
   size_t b = sizeof(double) * M;
   b += sizeof(float) * ((size_t)block_q * d + 2 * (size_t)block_q + 2 * (size_t)M +
@@ -361,6 +363,8 @@ size_t attend_smem_bytes(int d, int M, int C, int P, int block_q) {
   b += sizeof(int) * ((size_t)M + (size_t)(P > 0 ? P : 1));
   return b;
 }
+
+namespace {
 
 template <typename T>
 avq_status launch_assign(const avq_problem& p, const void* K, const void* Cp, const void* Cc,
@@ -388,8 +392,8 @@ avq_status launch_aggregate(const avq_problem& p, const void* V, const int32_t* 
 
 template <typename T>
 avq_status launch_attend(const AttendArgs& a, int B, cudaStream_t st) {
-  const size_t smem = attend_smem_bytes(a.d, a.M, a.C, a.P, a.block_q);
-  if (smem > 200 * 1024) return AVQ_ERR_UNSUPPORTED;
+  const size_t smem = simt_attend_smem_bytes(a.d, a.M, a.C, a.P, a.block_q);
+  if (smem > kSimtAttendSmemLimit) return AVQ_ERR_UNSUPPORTED;   // validate_forward rejects these up front
   auto kern = attend_simt_kernel<T>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return AVQ_ERR_CUDA;

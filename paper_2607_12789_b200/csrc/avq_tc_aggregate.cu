@@ -2,9 +2,11 @@
 //
 // leaf_scatter_kernel  one warp per 8 keys: each key's V row is added to the sum of its leaf
 //                      codeword (parent, child) with vector reductions to global memory, and
-//                      the leaf's count is bumped.  Only the leaf level is scattered.
-// finalize_kernel      per parent: Vp = sum over its children (every key sits in exactly one
-//                      child, so the parent sum is the sum of its leaves), np likewise, and
+//                      the leaf's count is bumped.  Only the leaf level is scattered; a key whose
+//                      child index is -1 (it stays with its parent, Algorithm 1's masked scatter)
+//                      goes to its parent's "stay" leaf, which is the parent's own row of Vp / np.
+// finalize_kernel      per parent: Vp = stay part + sum over its children (every key sits in
+//                      exactly one leaf, so the parent sum is the sum of its leaves), np likewise, and
 //                      the bf16 operand copies the attention kernel stages (rows = codewords, the
 //                      MN-major B operand of its value MMAs):
 //                        Vpb [B,H,M,d]    parent value sums
@@ -26,7 +28,8 @@ template <int D>
 __global__ void __launch_bounds__(kScatterThreads)
 leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restrict__ pidx,
                     const int32_t* __restrict__ cidx, float* __restrict__ Vc, float* __restrict__ nc,
-                    int Nk, int M, int C) {
+                    float* __restrict__ Vp, float* __restrict__ np_, int Nk, int M, int C,
+                    int32_t* status_word) {
   tc::pdl_launch_dependents();
   const int bh = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -48,24 +51,36 @@ leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restri
   }
   tc::pdl_wait();                                    // the indices come from the kernel before
   if (j0 >= Nk) return;
+  // an earlier kernel of this call gave up on a wait: its indices are not valid, do not scatter them
+  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word) != 0) return;
+  // leaf_l: a * C + c for a key that moved to child c, kStayBit | a for a key that stays, -1 = nothing to add
+  constexpr int kStayBit = 1 << 30;
   int leaf_l = -1;
   if (lane < kKeysPerWarp && j0 + lane < Nk) {
     const int a = __ldg(pidx + kb + j0 + lane);
     const int c = __ldg(cidx + kb + j0 + lane);
-    leaf_l = a * C + c;
+    if (a < 0 || a >= M || c < -1 || c >= C) {       // caller-supplied index out of range: skip the key, flag it
+      if (status_word) atomicCAS(status_word, 0, DEV_BAD_INDEX);
+    } else {
+      leaf_l = c < 0 ? (kStayBit | a) : a * C + c;
+    }
   }
 #pragma unroll
   for (int t = 0; t < kSteps; ++t) {
     const int leaf = __shfl_sync(0xffffffffu, leaf_l, t * kRowsPerStep + sub);
     if (leaf >= 0) {
-      float* dst = Vc + ((size_t)bh * M * C + leaf) * D;
+      float* dst = (leaf & kStayBit) ? Vp + ((size_t)bh * M + (leaf & ~kStayBit)) * D
+                                     : Vc + ((size_t)bh * M * C + leaf) * D;
       const uint2 u = v[t];
       atomicAdd(reinterpret_cast<float4*>(dst) + col,
                 make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u),
                             __uint_as_float(u.y << 16), __uint_as_float(u.y & 0xFFFF0000u)));
     }
   }
-  if (leaf_l >= 0) atomicAdd(nc + (size_t)bh * M * C + leaf_l, 1.0f);
+  if (leaf_l >= 0) {
+    if (leaf_l & kStayBit) atomicAdd(np_ + (size_t)bh * M + (leaf_l & ~kStayBit), 1.0f);
+    else atomicAdd(nc + (size_t)bh * M * C + leaf_l, 1.0f);
+  }
 }
 
 // Long sequences over few codewords put hundreds of keys on every leaf, and the reductions above then
@@ -76,7 +91,7 @@ leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restri
 constexpr int kSortThreads = 512;
 constexpr int kSortKeysPerThread = 16;
 constexpr int kSortMaxKeys = kSortThreads * kSortKeysPerThread;   // keys per CTA (16-bit key field of the order list)
-constexpr int kSortMaxLeaves = 2048;                              // M * C <= 256 * 8
+constexpr int kSortMaxLeaves = 256 * 9;                           // M * (C + 1) <= 256 * 9: C children + the stay leaf
 // The chunked variant is chosen for heads of at least kSortMinKeys keys when a CTA's chunk holds at least
 // 0.8 keys per leaf (measured: faster from there on; short heads leave its 512-thread CTAs idle).
 constexpr int kSortRatio10 = 8;
@@ -86,7 +101,10 @@ template <int D>
 __global__ void __launch_bounds__(kSortThreads, 2)
 leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restrict__ pidx,
                    const int32_t* __restrict__ cidx, float* __restrict__ Vc, float* __restrict__ nc,
-                   int Nk, int L, int C, int chunk) {
+                   float* __restrict__ Vp, float* __restrict__ np_, int Nk, int M, int C, int chunk,
+                   int32_t* status_word) {
+  // leaves of a parent: its C children, then (index C) the keys that stay with the parent itself
+  const int C1 = C + 1, L = M * C1;
   extern __shared__ __align__(16) unsigned char sort_smem[];
   int* hist = reinterpret_cast<int*>(sort_smem);        // [L] keys per leaf
   int* offs = hist + L;                                 // [L] first slot of each leaf in `order`
@@ -101,6 +119,8 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
   __syncthreads();
   tc::pdl_wait();                                      // the indices come from the kernel before
   if (n <= 0) return;
+  // an earlier kernel of this call gave up on a wait: its indices are not valid, do not scatter them
+  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word) != 0) return;
   const size_t kb = (size_t)bh * Nk + j0;
 
   // ---- leaf of every key and its rank among the chunk's keys of that leaf
@@ -110,22 +130,30 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
     const int j = tid + t * kSortThreads;
     lr[t] = 0xFFFFFFFFu;
     if (j < n) {
-      const int leaf = __ldg(pidx + kb + j) * C + __ldg(cidx + kb + j);
-      lr[t] = ((uint32_t)leaf << 16) | (uint32_t)atomicAdd(&hist[leaf], 1);
+      const int a = __ldg(pidx + kb + j), c = __ldg(cidx + kb + j);
+      if (a < 0 || a >= M || c < -1 || c >= C) {       // caller-supplied index out of range: skip the key, flag it
+        if (status_word) atomicCAS(status_word, 0, DEV_BAD_INDEX);
+      } else {
+        const int leaf = a * C1 + (c < 0 ? C : c);
+        lr[t] = ((uint32_t)leaf << 16) | (uint32_t)atomicAdd(&hist[leaf], 1);
+      }
     }
   }
   __syncthreads();
 
   // ---- exclusive scan of the histogram: thread t owns entries [t * E, (t + 1) * E); key counts go out
   {
-    const int E = (L + kSortThreads - 1) / kSortThreads;   // <= 4
-    int c[4] = {0, 0, 0, 0}, tot = 0;
+    const int E = (L + kSortThreads - 1) / kSortThreads;   // <= 5
+    int c[5] = {0, 0, 0, 0, 0}, tot = 0;
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
+    for (int e = 0; e < 5; ++e)
       if (e < E && tid * E + e < L) {
         c[e] = hist[tid * E + e];
         tot += c[e];
-        if (c[e] > 0) atomicAdd(nc + (size_t)bh * L + tid * E + e, (float)c[e]);
+        if (c[e] > 0) {
+          const int leaf = tid * E + e, a = leaf / C1, cc = leaf - a * C1;
+          atomicAdd(cc == C ? np_ + (size_t)bh * M + a : nc + ((size_t)bh * M + a) * C + cc, (float)c[e]);
+        }
       }
     int inc = tot;
 #pragma unroll
@@ -138,7 +166,7 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
     int base = inc - tot;
     for (int u = 0; u < warp; ++u) base += wsum[u];
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
+    for (int e = 0; e < 5; ++e)
       if (e < E && tid * E + e < L) { offs[tid * E + e] = base; base += c[e]; }
   }
   __syncthreads();
@@ -153,13 +181,15 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
   using Word = typename std::conditional<D == 64, uint32_t, uint2>::type;
   const Word* Vw = reinterpret_cast<const Word*>(V + kb * D) + lane;   // row j at Vw + j * 32
   constexpr int kWarps = kSortThreads / 32, kBatch = 16;
-  const int share = (n + kWarps - 1) / kWarps;
-  const int s0 = warp * share, s1 = min(n, s0 + share);
+  const int listed = offs[L - 1] + hist[L - 1];         // keys in the ordered list (= n unless some were skipped)
+  const int share = (listed + kWarps - 1) / kWarps;
+  const int s0 = warp * share, s1 = min(listed, s0 + share);
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
   int cur = -1;
   auto flush = [&]() {
     if (cur < 0) return;
-    float* dst = Vc + ((size_t)bh * L + cur) * D;
+    const int a = cur / C1, cc = cur - a * C1;
+    float* dst = cc == C ? Vp + ((size_t)bh * M + a) * D : Vc + (((size_t)bh * M + a) * C + cc) * D;
     if constexpr (D == 64) atomicAdd(reinterpret_cast<float2*>(dst) + lane, make_float2(acc[0], acc[1]));
     else atomicAdd(reinterpret_cast<float4*>(dst) + lane, make_float4(acc[0], acc[1], acc[2], acc[3]));
     acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
@@ -206,9 +236,10 @@ template <int D, int C>
 __global__ void __launch_bounds__(D)
 finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, float* __restrict__ Vp,
                 float* __restrict__ np_, __nv_bfloat16* __restrict__ Vpb, __nv_bfloat16* __restrict__ Vcb,
-                int M) {
+                int M, const int32_t* status_word) {
   tc::pdl_launch_dependents();
   tc::pdl_wait();                                    // the leaf sums come from the kernel before
+  if (status_word && *reinterpret_cast<const volatile int32_t*>(status_word) != 0) return;
   const int bh = blockIdx.y, m0 = blockIdx.x * 8, k = threadIdx.x;
   constexpr int kPer = (C == 4) ? 8 : 4;             // parents whose loads are in flight together (32 floats)
 #pragma unroll
@@ -222,7 +253,7 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
 #pragma unroll
     for (int mm = 0; mm < kPer; ++mm) {
       const size_t row = (size_t)bh * M + m0 + g * kPer + mm;
-      float s = 0.f;
+      float s = Vp[row * D + k];                       // the stay part, accumulated by the scatter (zero by default)
 #pragma unroll
       for (int c = 0; c < C; ++c) {
         s += x[mm][c];
@@ -234,7 +265,7 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
   }
   if (k < 8) {
     const int m = m0 + k;
-    float s = 0.f;
+    float s = np_[(size_t)bh * M + m];                 // keys that stay with the parent
 #pragma unroll
     for (int c = 0; c < C; ++c) s += nc[((size_t)bh * M + m) * C + c];
     np_[(size_t)bh * M + m] = s;
@@ -243,11 +274,14 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
 
 template <int D, int C>
 avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const int32_t* cidx, float* Vp,
-               float* np_, float* Vc, float* nc, void* Vpb, void* Vcb, bool pre_zeroed, cudaStream_t st) {
+               float* np_, float* Vc, float* nc, void* Vpb, void* Vcb, bool pre_zeroed, int32_t* status_word,
+               cudaStream_t st) {
   const unsigned BH = (unsigned)(p.B * p.H);
   if (!pre_zeroed) {
     if (cudaMemsetAsync(Vc, 0, sizeof(float) * (size_t)BH * p.M * C * D, st) != cudaSuccess) return AVQ_ERR_CUDA;
     if (cudaMemsetAsync(nc, 0, sizeof(float) * (size_t)BH * p.M * C, st) != cudaSuccess) return AVQ_ERR_CUDA;
+    if (cudaMemsetAsync(Vp, 0, sizeof(float) * (size_t)BH * p.M * D, st) != cudaSuccess) return AVQ_ERR_CUDA;
+    if (cudaMemsetAsync(np_, 0, sizeof(float) * (size_t)BH * p.M, st) != cudaSuccess) return AVQ_ERR_CUDA;
   }
   // `pre_zeroed` marks the chained call from avq_forward: the kernel before in the stream is the assign
   // kernel, so the scatter may be launched as its programmatic dependent.
@@ -271,7 +305,7 @@ avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const i
   chunk = (chunk + 31) & ~31;
   if (L <= kSortMaxLeaves && p.Nk >= kSortMinKeys && chunk * 10 >= kSortRatio10 * L) {
     dim3 g1((p.Nk + chunk - 1) / chunk, BH);
-    const size_t smem = sizeof(int) * (2 * (size_t)L + 16) + sizeof(uint32_t) * (size_t)chunk;
+    const size_t smem = sizeof(int) * (2 * (size_t)p.M * (C + 1) + 16) + sizeof(uint32_t) * (size_t)chunk;
     // above the default limit only for the largest leaf count and chunk: opt in once per device
     static bool configured[64] = {};
     int dev = 0;
@@ -284,30 +318,32 @@ avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const i
       if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     if (tc::launch_pdl(leaf_sorted_kernel<D>, g1, dim3(kSortThreads), smem, st, pre_zeroed,
-                       static_cast<const __nv_bfloat16*>(V), pidx, cidx, Vc, nc, p.Nk, L, C, chunk) != cudaSuccess)
+                       static_cast<const __nv_bfloat16*>(V), pidx, cidx, Vc, nc, Vp, np_, p.Nk, p.M, C, chunk,
+                       status_word) != cudaSuccess)
       return AVQ_ERR_CUDA;
   } else {
     dim3 g1((p.Nk + kKeysPerCta - 1) / kKeysPerCta, BH);
     if (tc::launch_pdl(leaf_scatter_kernel<D>, g1, dim3(kScatterThreads), 0, st, pre_zeroed,
-                       static_cast<const __nv_bfloat16*>(V), pidx, cidx, Vc, nc, p.Nk, p.M, C) != cudaSuccess)
+                       static_cast<const __nv_bfloat16*>(V), pidx, cidx, Vc, nc, Vp, np_, p.Nk, p.M, C,
+                       status_word) != cudaSuccess)
       return AVQ_ERR_CUDA;
   }
   dim3 g2(p.M / 8, BH);
   return cuda_ok(tc::launch_pdl(finalize_kernel<D, C>, g2, dim3(D), 0, st, true, static_cast<const float*>(Vc),
                                 static_cast<const float*>(nc), Vp, np_, static_cast<__nv_bfloat16*>(Vpb),
-                                static_cast<__nv_bfloat16*>(Vcb), p.M));
+                                static_cast<__nv_bfloat16*>(Vcb), p.M, static_cast<const int32_t*>(status_word)));
 }
 
 }  // namespace
 
 avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
                         const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc, void* Vpb,
-                        void* Vcb, bool pre_zeroed, cudaStream_t st) {
+                        void* Vcb, bool pre_zeroed, int32_t* status_word, cudaStream_t st) {
   if (p.d == 64)
-    return p.C == 4 ? run<64, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, st)
-                    : run<64, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, st);
-  return p.C == 4 ? run<128, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, st)
-                  : run<128, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, st);
+    return p.C == 4 ? run<64, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, status_word, st)
+                    : run<64, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, status_word, st);
+  return p.C == 4 ? run<128, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, status_word, st)
+                  : run<128, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, status_word, st);
 }
 
 }  // namespace avq

@@ -24,14 +24,6 @@ constexpr int kThreadsA = 256;
 // memory, at most 128 TMEM columns up to M = 128) for four to share an SM.
 constexpr int assign_min_ctas(int D, int NL) { return D == 64 ? 4 : 2; }
 
-#ifdef AVQ_PHASE_DEBUG
-__device__ long long g_assign_clocks[64 * 16];
-#define APHASE(i) do { if (threadIdx.x == 0 && blockIdx.x < 8 && blockIdx.y < 8) \
-    g_assign_clocks[(blockIdx.y * 8 + blockIdx.x) * 16 + (i)] = clock64(); } while (0)
-#else
-#define APHASE(i) do { } while (0)
-#endif
-
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
 
@@ -110,8 +102,6 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   const int bh = blockIdx.y, h = bh % H;
   const int j0 = blockIdx.x * kKeys;
   const int MH = M >> 1;                             // columns per half (multiple of 16: M % 32 == 0)
-
-  APHASE(0);
   pdl_launch_dependents();   // the next kernel of the call may begin its set-up
   // Inside avq_forward the grid also clears the accumulators of the aggregation that follows (status
   // header, leaf sums, leaf counts: zero_units 16-byte words), each CTA an equal slice; the stores drain
@@ -145,10 +135,8 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  APHASE(1);
 
   const bool loaded = mbar_wait(&bars[0], 0, abort_flag, status_word, DEV_TIMEOUT_ASSIGN);
-  APHASE(2);
   if (tid == 0 && loaded) {
     tc_fence_after();
     const uint32_t idesc = umma_idesc_bf16(kKeys, M);
@@ -195,13 +183,10 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     }
     xkn[hf * kKeys + r] = s;
   }
-  APHASE(3);
   __syncthreads();   // cnorm, cmax visible
-  APHASE(4);
 
   const bool done = mbar_wait(&bars[1], 0, abort_flag, status_word, DEV_TIMEOUT_ASSIGN);
   tc_fence_after();
-  APHASE(5);
 
   // ---- parent argmin over this thread's half of the columns
   {
@@ -228,11 +213,9 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     xd2[hf * kKeys + r] = d2;
     xi1[hf * kKeys + r] = i1;
   }
-  APHASE(6);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
-  APHASE(7);
 
   // ---- merge the halves (the lower half holds the lower indices, so it wins ties); recheck near-ties
   const __nv_bfloat16* Cph = Cp + (size_t)h * M * D;
@@ -257,7 +240,6 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     par[r] = i1;
   }
   __syncthreads();
-  APHASE(8);
 
   {
     // ---- child argmin, four lanes per key: a warp takes 8 keys at a time (two passes over its 16 keys).
@@ -342,12 +324,13 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     }
   }
   __syncthreads();
-  APHASE(9);
-  if (tid < kKeys && j0 + tid < Nk && done) {
+  // When a wait above gave up the indices are meaningless, but they are in range (both argmins start
+  // from index 0 and only take loop indices), so the kernels behind this one read nothing out of bounds;
+  // they see the recorded status word and skip their work.
+  if (tid < kKeys && j0 + tid < Nk) {
     pidx[(size_t)bh * Nk + j0 + tid] = par[tid];
     cidx[(size_t)bh * Nk + j0 + tid] = chi[tid];
   }
-  APHASE(10);
 }
 
 uint32_t pow2_cols(int n) {
@@ -395,12 +378,6 @@ avq_status launch(const avq_problem& p, const void* K, const void* Cp, const voi
 }
 
 }  // namespace
-
-#ifdef AVQ_PHASE_DEBUG
-extern "C" __attribute__((visibility("default"))) int avq_debug_assign_clocks(long long* host_out) {
-  return (int)cudaMemcpyFromSymbol(host_out, g_assign_clocks, sizeof(long long) * 64 * 16);
-}
-#endif
 
 avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const void* Cc,
                      int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, void* zero_base,

@@ -90,22 +90,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, ui
   return ok != 0;
 }
 // Bounded wait: each try suspends for a few microseconds at most; after every failed try the abort flag
-// and the clock are looked at; gives up after kWaitLimitNs or kWaitLimitPolls tries.  Returns false (and
-// flags the failure) when it gives up or when the CTA has already aborted.
+// and the clock are looked at; gives up after the time limit (kWaitLimitNs unless the caller gives its own)
+// or after kWaitLimitPolls = 2^22 tries.  Returns false (and flags the failure) when it gives up or when
+// the CTA has already aborted.
 constexpr uint32_t kWaitLimitPolls = 1u << 22;
 constexpr uint32_t kWaitTryNs = 4000;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* status_word, int32_t code) {
+__device__ __forceinline__ bool mbar_wait_for(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                              int32_t* status_word, int32_t code, unsigned long long limit_ns) {
   if (mbar_test_wait(bar, parity)) return true;
   const unsigned long long t0 = global_timer_ns();
   for (uint32_t polls = 0; polls < kWaitLimitPolls; ++polls) {
     if (mbar_try_wait(bar, parity, kWaitTryNs)) return true;
     if (*abort_flag) return false;
-    if (global_timer_ns() - t0 > kWaitLimitNs) break;
+    if (global_timer_ns() - t0 > limit_ns) break;
   }
   *abort_flag = 1;
   if (status_word) atomicCAS(status_word, 0, code);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status_word, int32_t code) {
+  return mbar_wait_for(bar, parity, abort_flag, status_word, code, kWaitLimitNs);
 }
 
 // Asynchronous global -> shared copies that bypass registers (generic proxy; follow the wait with

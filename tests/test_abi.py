@@ -28,8 +28,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_status_strings(lib):
-    seen = {lib.avq_status_string(s).decode() for s in range(8)}
-    assert len(seen) == 8 and "ok" in seen
+    seen = {lib.avq_status_string(s).decode() for s in range(9)}
+    assert len(seen) == 9 and "ok" in seen
     assert lib.avq_status_string(99).decode() == "unknown status"
 
 
@@ -58,6 +58,7 @@ def test_workspace_bytes_and_layout(lib):
     (dict(), 17, 64, 2), (dict(), -1, 64, 2), (dict(), 2, 0, 2), (dict(scale=float("nan")), 2, 64, 2),
     (dict(d=6), 2, 64, 3), (dict(d=512), 2, 64, 3), (dict(M=2048), 2, 64, 3), (dict(C=32), 2, 64, 3),
     (dict(), 2, 512, 3), (dict(B=70000), 2, 64, 3),
+    (dict(d=256), 2, 256, 3),                                   # CUDA-core attention tile beyond 200 KiB of shared memory
     (dict(dtype_code=binding.AVQ_BF16, d=96), 2, 128, 3), (dict(dtype_code=binding.AVQ_BF16, M=24), 2, 128, 3),
     (dict(dtype_code=binding.AVQ_BF16, C=3), 2, 128, 3), (dict(dtype_code=binding.AVQ_BF16), 2, 64, 3),
     (dict(dtype_code=binding.AVQ_BF16, flags=binding.FLAG_PARENT_STAYS), 2, 128, 3),

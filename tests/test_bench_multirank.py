@@ -40,3 +40,27 @@ def test_two_gloo_ranks_share_nothing_but_the_step_time():
 def test_single_rank_needs_no_process_group():
     import bench
     assert bench.max_over_ranks(2.5, 1, torch.device("cpu")) == 2.5
+
+
+def test_timed_loop_is_repeated_until_enough_time_is_covered():
+    import bench
+    assert bench.repeats_for(5.6) == 36                        # 20 steps of 0.28 ms: 36 repeats reach 200 ms
+    assert bench.repeats_for(500.0) == 1
+    assert bench.repeats_for(1e-4) == bench.MAX_REPEATS
+
+
+def test_recorded_dram_traffic_is_dropped_when_the_kernel_sources_changed(tmp_path, monkeypatch):
+    import json
+    import bench
+    from paper_2607_12789_b200 import build
+    prof = tmp_path / "profiles"
+    prof.mkdir()
+    rec = dict(source_hash=build.source_hash(), command="ncu ...",
+               entries=[dict(workload="c3_long", kernel="attend", dram_bytes_per_launch=1.0e8)])
+    (prof / "ncu_traffic.json").write_text(json.dumps(rec))
+    monkeypatch.setattr(bench, "ROOT", str(tmp_path))
+    assert bench.measured_traffic("c3_long", "attend")[0] == 1.0e8
+    assert bench.measured_traffic("c1_vitb", "attend")[0] is None
+    rec["source_hash"] = "0" * 16
+    (prof / "ncu_traffic.json").write_text(json.dumps(rec))
+    assert bench.measured_traffic("c3_long", "attend")[0] is None

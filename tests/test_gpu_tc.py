@@ -36,25 +36,75 @@ def test_c3_long_sampled():
     assert np.array_equal(gpu["nc"].sum(axis=-1), gpu["np"])
     np.testing.assert_allclose(gpu["importance"].sum(axis=-1), 128.0, rtol=1e-4)
     np.testing.assert_allclose(gpu["Vp"].sum(axis=2), x["V"].astype(np.float64).sum(axis=2), atol=5e-3)
+    # every query tile of six heads against the factorised oracle (768 of the 2048 tiles)
+    rep2, _ = parity.heads_parity_factorised(synth.C3, [(0, h) for h in (0, 3, 6, 9, 12, 15)], x=x, gpu=gpu)
+    print("c3 whole heads", rep2)
+    assert rep2["blocks"] >= 6 * 128 - rep2["topp_flips_excused"]
 
 
+# Sweep configuration: every (N, M, P) point has a parity test.  All P of one (N, M) share their data, so
+# the oracle's assignment of a head is computed once per (N, M).  N <= 16384: every query tile of the
+# listed heads (factorised oracle); N = 65536: one head, every tile.
 @pytest.mark.parametrize("M", [32, 64, 128, 256])
 def test_sweep_N1024_all_P(M):
     for P in synth.sweep_P(M):
         parity.full_parity(synth.sweep_point(1024, M, P).with_(H=4))
 
 
-@pytest.mark.parametrize("M,P", [(64, 16), (256, 64), (128, 128)])
-def test_sweep_N4096(M, P):
-    parity.full_parity(synth.sweep_point(4096, M, P).with_(H=2))
+@pytest.mark.parametrize("M", [32, 64, 128, 256])
+@pytest.mark.parametrize("N,H", [(4096, 2), (16384, 1), (65536, 1)])
+def test_sweep_all_P_whole_heads(N, H, M):
+    wl0 = synth.sweep_point(N, M, 0).with_(H=H)
+    x = synth.generate(wl0)
+    heads = [(0, h) for h in range(H)]
+    cache = {}
+    for P in synth.sweep_P(M):
+        rep, cache = parity.heads_parity_factorised(wl0.with_(P=P), heads, x=x, assignments=cache, P=P)
+        print(f"sweep N={N} M={M} P={P}", rep)
 
 
-def test_sweep_N16384_sampled():
+def test_sweep_dense_definition_on_sampled_tiles():
+    """The O(N^2) definition itself on sampled tiles of long sweep points."""
     parity.sampled_parity(synth.sweep_point(16384, 256, 32), heads=[(0, 5)], blocks_per_head=6)
-
-
-def test_sweep_N65536_sampled():
     parity.sampled_parity(synth.sweep_point(65536, 64, 16), heads=[(0, 9)], blocks_per_head=4)
+
+
+def _exact_grid(g, shape, step=0.25, lim=4.0):
+    """Random values on a coarse grid: exactly representable in bf16, sums of squares exact in fp32."""
+    return (np.clip(np.round(g.normal(size=shape) / step), -lim / step, lim / step) * step).astype(np.float32)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("C", [4, 8])
+def test_exact_ties_on_the_tensor_core_path(d, C):
+    """Duplicated parent codewords, duplicated children, keys at exact midpoints and keys equal to
+    codewords, inside the tcgen05 envelope (M = 32): best and runner-up distances coincide, so the
+    float64 recheck of avq_assign decides, and the lowest index must win (Algorithm 1's strict '<')."""
+    from oracle import avq_oracle as orc
+    g = np.random.default_rng(7 + d + C)
+    M = 32
+    base = _exact_grid(g, (12, d))
+    Cp = base[g.integers(0, 12, size=M)]                      # 32 parents drawn from 12 distinct rows
+    Cp[5] = Cp[2]; Cp[9] = Cp[2]; Cp[31] = Cp[30]
+    Cc = np.repeat(Cp[:, None, :], C, axis=1).copy()
+    Cc[:, C // 2:] += 0.5                                     # children 0..C/2-1 equal, C/2..C-1 equal
+    Cc[3] = _exact_grid(g, (C, d))
+    Cc[3, 2] = Cc[3, 1]                                       # a duplicated pair in the middle
+    keys = [Cp,                                               # keys on parent codewords
+            Cc.reshape(-1, d),                                # keys on child codewords
+            0.5 * (Cp[:16] + Cp[16:]),                        # exact midpoints of two parents
+            0.5 * (Cc[:, 0] + Cc[:, C - 1]),                  # exact midpoints of two children
+            _exact_grid(g, (200, d))]
+    K = np.concatenate(keys).astype(np.float32)
+    assert np.array_equal(synth.round_to_bf16(K), K) and np.array_equal(synth.round_to_bf16(Cc), Cc)
+    ref = orc.assign_head(K, Cp, Cc)
+    assert (ref["parent_margin"] == 0).sum() >= M and (ref["child_margin"] == 0).sum() >= M
+    assert ref["parent_idx"][5] == 2 and ref["parent_idx"][9] == 2 and ref["parent_idx"][31] == 30
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda().to(torch.bfloat16)
+    pi, ci = binding.assign(t(K[None, None]), t(Cp[None]), t(Cc[None]))
+    torch.cuda.synchronize()
+    assert np.array_equal(pi.cpu().numpy()[0, 0], ref["parent_idx"])
+    assert np.array_equal(ci.cpu().numpy()[0, 0], ref["child_idx"])
 
 
 def test_ragged_tail_and_nq_not_nk():

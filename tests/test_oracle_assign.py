@@ -103,6 +103,24 @@ def test_midpoint_key_is_a_tie_resolved_to_lower_index():
     assert got["child_idx"][0] == 0 and got["child_margin"][0] == 0.0
 
 
+def test_stay_margin_is_the_relative_gap_between_child_and_parent_distance():
+    """One parent at the origin with children at x = 3 and x = -5 (1-d keys written out by hand):
+    key 1.0 -> parent distance 1, nearest child distance 4, margin (4 - 1) / 4 = 0.75, the key stays;
+    key 2.0 -> 4 vs 1, margin 0.75, the key moves; key 1.5 -> 2.25 vs 2.25: margin 0, strict '<' keeps
+    it with the parent; key 0 on the parent -> 0 vs 9, margin 1."""
+    Cp = np.array([[0.0]])
+    Cc = np.array([[[3.0], [-5.0]]])
+    K = np.array([[1.0], [2.0], [1.5], [0.0]])
+    got = orc.assign_head(K, Cp, Cc, parent_stays=True)
+    np.testing.assert_allclose(got["d_parent"], [1.0, 4.0, 2.25, 0.0], rtol=0, atol=0)
+    np.testing.assert_allclose(got["d_child"], [4.0, 1.0, 2.25, 9.0], rtol=0, atol=0)
+    np.testing.assert_allclose(got["stay_margin"], [0.75, 0.75, 0.0, 1.0], rtol=0, atol=1e-15)
+    assert got["child_idx"].tolist() == [-1, 0, -1, -1]
+    rep = orc.assign_head(K, Cp, Cc, parent_stays=False)
+    assert rep["child_idx"].tolist() == [0, 0, 0, 0]
+    np.testing.assert_allclose(rep["stay_margin"], got["stay_margin"])
+
+
 def test_replace_and_parent_stays_differ_only_where_the_parent_is_closer():
     w = synth.C0.with_(keys_around_parents=True, sigma_k=0.05)
     x = synth.generate(w)

@@ -45,3 +45,16 @@ def test_static_workspace_matches_caller_workspace_twice_in_a_row(wl):
         assert (Y.float() - Y_ref.float()).abs().max().item() <= tol
         assert torch.equal(topp, topp_ref)
         assert torch.allclose(imp, imp_ref, rtol=1e-4, atol=1e-5)
+    # the entry point itself allocates nothing: free device memory is the same before and after a call
+    # whose outputs already exist (the caching allocator is not involved: raw ctypes call, own buffers)
+    prob = binding._problem_from(dv["Q"], dv["K"], dv["Cp"], dv["Cc"], wl.scale, 0)
+    Y2 = torch.empty_like(dv["Q"])
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    st = binding.lib().avq_forward_static(ctypes.byref(prob), binding._ptr(dv["Q"]), binding._ptr(dv["K"]),
+                                          binding._ptr(dv["V"]), binding._ptr(dv["Cp"]), binding._ptr(dv["Cc"]),
+                                          wl.P, wl.block_q, binding._ptr(Y2), None, None, binding._stream())
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert st == 0 and free_after == free_before
+    assert (Y2.float() - Y_ref.float()).abs().max().item() <= tol
