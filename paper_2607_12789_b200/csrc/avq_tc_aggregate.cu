@@ -7,10 +7,11 @@
 //                      goes to its parent's "stay" leaf, which is the parent's own row of Vp / np.
 // finalize_kernel      per parent: Vp = stay part + sum over its children (every key sits in
 //                      exactly one leaf, so the parent sum is the sum of its leaves), np likewise, and
-//                      the bf16 operand copies the attention kernel stages (rows = codewords, the
-//                      MN-major B operand of its value MMAs):
-//                        Vpb [B,H,M,d]    parent value sums
-//                        Vcb [B,H,M,C,d]  leaf value sums: a parent's C children are C consecutive rows
+//                      the bf16 operands the attention kernel stages (rows = codewords, the
+//                      MN-major B operand of its value MMAs), as per-codeword MEANS (sum / count, zero
+//                      for an empty codeword):
+//                        Vpb [B,H,M,d]    parent value means
+//                        Vcb [B,H,M,C,d]  leaf value means: a parent's C children are C consecutive rows
 #include <type_traits>
 
 #include "avq_tc_common.cuh"
@@ -254,15 +255,20 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
     for (int mm = 0; mm < kPer; ++mm) {
       const size_t row = (size_t)bh * M + m0 + g * kPer + mm;
       float s = Vp[row * D + k];                       // the stay part, accumulated by the scatter (zero by default)
+      float n = np_[row];                              // keys that stay (the total is written after the barrier below)
 #pragma unroll
       for (int c = 0; c < C; ++c) {
+        const float ncc = nc[row * C + c];
         s += x[mm][c];
-        if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(x[mm][c]);
+        n += ncc;
+        // the attention kernel takes per-codeword MEANS: the count rides in its softmax weight
+        if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(ncc > 0.f ? x[mm][c] / ncc : 0.f);
       }
       Vp[row * D + k] = s;
-      if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(s);
+      if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(n > 0.f ? s / n : 0.f);
     }
   }
+  __syncthreads();                                     // every thread has read the stay counts
   if (k < 8) {
     const int m = m0 + k;
     float s = np_[(size_t)bh * M + m];                 // keys that stay with the parent

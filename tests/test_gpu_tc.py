@@ -99,7 +99,10 @@ def test_exact_ties_on_the_tensor_core_path(d, C):
     assert np.array_equal(synth.round_to_bf16(K), K) and np.array_equal(synth.round_to_bf16(Cc), Cc)
     ref = orc.assign_head(K, Cp, Cc)
     assert (ref["parent_margin"] == 0).sum() >= M and (ref["child_margin"] == 0).sum() >= M
-    assert ref["parent_idx"][5] == 2 and ref["parent_idx"][9] == 2 and ref["parent_idx"][31] == 30
+    # a key that sits on parent i must be given the FIRST parent with that codeword (written out by hand)
+    first_equal = [min(j for j in range(M) if np.array_equal(Cp[j], Cp[i])) for i in range(M)]
+    assert ref["parent_idx"][:M].tolist() == first_equal and first_equal[5] == first_equal[9] == first_equal[2]
+    assert len(set(first_equal)) <= 12
     t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda().to(torch.bfloat16)
     pi, ci = binding.assign(t(K[None, None]), t(Cp[None]), t(Cc[None]))
     torch.cuda.synchronize()
