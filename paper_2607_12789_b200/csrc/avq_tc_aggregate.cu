@@ -104,8 +104,8 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
                    const int32_t* __restrict__ cidx, float* __restrict__ Vc, float* __restrict__ nc,
                    float* __restrict__ Vp, float* __restrict__ np_, int Nk, int M, int C, int chunk,
                    int32_t* status_word) {
-  // leaves of a parent: its C children, then (index C) the keys that stay with the parent itself
-  const int C1 = C + 1, L = M * C1;
+  // leaves: (parent, child) pairs at a * C + c, then one "stay" leaf per parent at M * C + a
+  const int MC = M * C, L = MC + M;
   extern __shared__ __align__(16) unsigned char sort_smem[];
   int* hist = reinterpret_cast<int*>(sort_smem);        // [L] keys per leaf
   int* offs = hist + L;                                 // [L] first slot of each leaf in `order`
@@ -135,7 +135,7 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
       if (a < 0 || a >= M || c < -1 || c >= C) {       // caller-supplied index out of range: skip the key, flag it
         if (status_word) atomicCAS(status_word, 0, DEV_BAD_INDEX);
       } else {
-        const int leaf = a * C1 + (c < 0 ? C : c);
+        const int leaf = c < 0 ? MC + a : a * C + c;
         lr[t] = ((uint32_t)leaf << 16) | (uint32_t)atomicAdd(&hist[leaf], 1);
       }
     }
@@ -152,8 +152,8 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
         c[e] = hist[tid * E + e];
         tot += c[e];
         if (c[e] > 0) {
-          const int leaf = tid * E + e, a = leaf / C1, cc = leaf - a * C1;
-          atomicAdd(cc == C ? np_ + (size_t)bh * M + a : nc + ((size_t)bh * M + a) * C + cc, (float)c[e]);
+          const int leaf = tid * E + e;
+          atomicAdd(leaf < MC ? nc + (size_t)bh * MC + leaf : np_ + (size_t)bh * M + (leaf - MC), (float)c[e]);
         }
       }
     int inc = tot;
@@ -189,8 +189,7 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
   int cur = -1;
   auto flush = [&]() {
     if (cur < 0) return;
-    const int a = cur / C1, cc = cur - a * C1;
-    float* dst = cc == C ? Vp + ((size_t)bh * M + a) * D : Vc + (((size_t)bh * M + a) * C + cc) * D;
+    float* dst = cur < MC ? Vc + ((size_t)bh * MC + cur) * D : Vp + ((size_t)bh * M + (cur - MC)) * D;
     if constexpr (D == 64) atomicAdd(reinterpret_cast<float2*>(dst) + lane, make_float2(acc[0], acc[1]));
     else atomicAdd(reinterpret_cast<float4*>(dst) + lane, make_float4(acc[0], acc[1], acc[2], acc[3]));
     acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
@@ -245,27 +244,32 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
   constexpr int kPer = (C == 4) ? 8 : 4;             // parents whose loads are in flight together (32 floats)
 #pragma unroll
   for (int g = 0; g < 8 / kPer; ++g) {
-    float x[kPer][C];
-#pragma unroll
-    for (int mm = 0; mm < kPer; ++mm)
-#pragma unroll
-      for (int c = 0; c < C; ++c)
-        x[mm][c] = Vc[((((size_t)bh * M + m0 + g * kPer + mm) * C) + c) * D + k];
+    // every load of the group is issued before the first use
+    float x[kPer][C], cn[kPer][C], stay[kPer], nstay[kPer];
 #pragma unroll
     for (int mm = 0; mm < kPer; ++mm) {
       const size_t row = (size_t)bh * M + m0 + g * kPer + mm;
-      float s = Vp[row * D + k];                       // the stay part, accumulated by the scatter (zero by default)
-      float n = np_[row];                              // keys that stay (the total is written after the barrier below)
 #pragma unroll
       for (int c = 0; c < C; ++c) {
-        const float ncc = nc[row * C + c];
+        x[mm][c] = Vc[(row * C + c) * D + k];
+        cn[mm][c] = nc[row * C + c];
+      }
+      stay[mm] = Vp[row * D + k];                      // accumulated by the scatter (zero unless keys stay)
+      nstay[mm] = np_[row];                            // keys that stay (the total is written after the barrier below)
+    }
+#pragma unroll
+    for (int mm = 0; mm < kPer; ++mm) {
+      const size_t row = (size_t)bh * M + m0 + g * kPer + mm;
+      float s = stay[mm], n = nstay[mm];
+#pragma unroll
+      for (int c = 0; c < C; ++c) {
         s += x[mm][c];
-        n += ncc;
-        // the attention kernel takes per-codeword MEANS: the count rides in its softmax weight
-        if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(ncc > 0.f ? x[mm][c] / ncc : 0.f);
+        n += cn[mm][c];
+        // the attention kernels take per-codeword MEANS: the count rides in their softmax weights
+        if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(cn[mm][c] > 0.f ? x[mm][c] * __frcp_rn(cn[mm][c]) : 0.f);
       }
       Vp[row * D + k] = s;
-      if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(n > 0.f ? s / n : 0.f);
+      if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(n > 0.f ? s * __frcp_rn(n) : 0.f);
     }
   }
   __syncthreads();                                     // every thread has read the stay counts

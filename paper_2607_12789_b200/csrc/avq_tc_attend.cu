@@ -36,7 +36,8 @@ constexpr int kParentWarps = 8;
 // warps 8..11 are the child warps (a warp reaches the TMEM lane quarter warp % 4)
 constexpr int kIssuerWarp = 12;
 constexpr int kSelectWarp = 13;
-constexpr int kAttendThreads = 14 * 32;
+constexpr int kLoaderWarp = 14;
+constexpr int kAttendThreads = 15 * 32;
 constexpr float kLazyLog2 = 8.f;        // a child maximum within 2^8 of the running one does not move it
 
 struct AttendParams {
@@ -73,7 +74,9 @@ enum Bar : int {
   B_PAIR = 19,      // [4] the two parent warps of a row quarter exchange (64 arrivals)
   B_PSYNC = 23,     // all parent threads (256 arrivals)
   B_DRAIN = 24,
-  B_COUNT = 25
+  B_QFREE = 25,     // [2] every MMA that read this Q buffer has completed (issuer -> loader)
+  B_XFREE = 27,     // the value tile's memory may take the next tile's values (issuer -> loader)
+  B_COUNT = 28
 };
 
 template <int D, int CT, int CHW, bool ALIAS>
@@ -264,6 +267,8 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     init(B_PAIR, 4, 64);
     init(B_PSYNC, 1, 32 * kParentWarps);
     init(B_DRAIN, 1, 1);
+    init(B_QFREE, 2, 1);
+    init(B_XFREE, 1, 1);
     mbar_fence_init();
     *abort_flag = 0;
     *early_exit = 0;
@@ -322,7 +327,6 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     umma_desc_sw128(cps + (k / 4) * M * 128 + (k % 4) * 32), idesc_s, k > 0);
         umma_commit(&bars[B_SFULL + (n & 1)]);
       };
-      issue_vp(t_begin / p.nblk);
       ok = AVQ_WAIT(B_QFULL, ph_q[0]) && AVQ_WAIT(B_CPFULL, ph_cp);
       ph_q[0] ^= 1;
       ph_cp ^= 1;
@@ -380,7 +384,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         ok = AVQ_WAIT(B_PVDONE, ph_pv);
         ph_pv ^= 1;
         if (!ok) break;
-        if (!ALIAS && has_next) issue_vp(bh_next);
+        if (!ALIAS && has_next) mbar_arrive(&bars[B_XFREE]);
         if (SB == 1 && has_next && !(ok = next_logits())) break;
 
         // ---- children of tile n
@@ -416,11 +420,8 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           ph_cpv[slot] ^= 1;
         }
         if (!ok) break;
-        if (ALIAS && has_next) issue_vp(bh_next);          // the child slots inside the value tile are free again
-        if (n + 2 < T) {
-          issue_q(n + 2);                                  // every MMA that read Q(n) has completed
-          if (n + 3 < T) prefetch_q(n + 3);
-        }
+        if (ALIAS && has_next) mbar_arrive(&bars[B_XFREE]);   // the child slots inside the value tile are free again
+        if (n + 2 < T) mbar_arrive(&bars[B_QFREE + (n & 1)]);  // every MMA that read Q(n) has completed
       }
       // every MMA issued above has completed on the normal path; after a failed wait give the ones in
       // flight (and the loads) time to finish before the CTA's shared memory and TMEM are released
@@ -429,6 +430,29 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (*abort_flag) {
         const unsigned long long t0 = global_timer_ns();
         while (global_timer_ns() - t0 < 100000ull) { }
+      }
+    }
+  } else if (warp == kLoaderWarp) {
+    // ================================================================ loader: the Q tiles and the value tiles
+    // (a TMA issue costs its thread several hundred cycles, which the MMA issuer cannot spare)
+    if (lane == 0) {
+      issue_vp(t_begin / p.nblk);
+      uint32_t ph_qf[2] = {0, 0}, ph_xf = 0;
+      bool ok = true;
+      for (int n = 0; ok && n < T; ++n) {
+        if (n + 1 < T) {
+          ok = AVQ_WAIT(B_XFREE, ph_xf);
+          ph_xf ^= 1;
+          if (!ok) break;
+          issue_vp((t_begin + n + 1) / p.nblk);
+        }
+        if (n + 2 < T) {
+          ok = AVQ_WAIT(B_QFREE + (n & 1), ph_qf[n & 1]);
+          ph_qf[n & 1] ^= 1;
+          if (!ok) break;
+          issue_q(n + 2);
+          if (n + 3 < T) prefetch_q(n + 3);
+        }
       }
     }
   } else if (warp < kParentWarps) {
@@ -565,12 +589,12 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         uint32_t thr = 0;
         bool exact = P >= M;                               // P = M: every parent (threshold 0, all keys reach it)
         if (!exact) {
+          // every lane forms the same count from ballots (no cross-lane reduction on the dependent path)
           for (int bit = 30; bit >= 0; --bit) {
             const uint32_t cand = thr | (1u << bit);
             int c = 0;
 #pragma unroll
-            for (int i = 0; i < NI; ++i) c += (key[i] >= cand) ? 1 : 0;
-            c = __reduce_add_sync(0xffffffffu, c);
+            for (int i = 0; i < NI; ++i) c += __popc(__ballot_sync(0xffffffffu, key[i] >= cand));
             if (c >= P) {
               thr = cand;
               if (c == P) { exact = true; break; }
@@ -581,8 +605,8 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (!exact) {
           int c = 0;
 #pragma unroll
-          for (int i = 0; i < NI; ++i) c += (key[i] > thr) ? 1 : 0;
-          need = P - __reduce_add_sync(0xffffffffu, c);   // places left for keys equal to the threshold
+          for (int i = 0; i < NI; ++i) c += __popc(__ballot_sync(0xffffffffu, key[i] > thr));
+          need = P - c;                                    // places left for keys equal to the threshold
         }
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
@@ -917,9 +941,13 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
 
 }  // namespace
 
+// Parent tiles of up to 128 codewords leave room for several small CTAs per SM (avq_tc_attend_small.cu);
+// larger ones take the whole SM and run the warp-specialised kernel above.
 avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc, const float* np_,
                      const float* nc, const void* Vpb, const void* Vcb, int32_t P, void* Y, int32_t* topp_out,
                      float* importance_out, int32_t* status_word, bool chained, cudaStream_t st) {
+  if (p.M <= 128)
+    return tc_attend_small(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, P, Y, topp_out, importance_out, status_word, chained, st);
   return p.d == 64 ? launch<64>(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, P, Y, topp_out, importance_out, status_word, chained, st)
                    : launch<128>(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, P, Y, topp_out, importance_out, status_word, chained, st);
 }
