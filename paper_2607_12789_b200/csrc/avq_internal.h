@@ -66,12 +66,6 @@ avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const 
                      void* Y, int32_t* topp_out, float* importance_out, int32_t* status_word,
                      bool chained, cudaStream_t st);   // chained: launched right behind tc_aggregate
 
-// the small-tile variant of tc_attend (M <= 128), same arguments
-avq_status tc_attend_small(const avq_problem& p, const void* Q, const void* Cp, const void* Cc,
-                           const float* np_, const float* nc, const void* Vpb, const void* Vcb, int32_t P,
-                           void* Y, int32_t* topp_out, float* importance_out, int32_t* status_word,
-                           bool chained, cudaStream_t st);
-
 inline avq_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? AVQ_OK : AVQ_ERR_CUDA; }
 
 }  // namespace avq

@@ -1,29 +1,23 @@
 // Tensor-core attention pass of AVQ-attention (Algorithm 2 in its masked form) for bf16 inputs.
 //
-// One persistent CTA per SM works through a contiguous run of query tiles (128 rows of one (batch, head)).
-// Its 14 warps have fixed roles, and two tiles are in flight: while the parent pass of tile n+1 runs on
-// the CUDA cores, the child pass and the output of tile n run beside it and the tensor pipe serves both.
-//
-//   issuer (1 warp, one lane)  TMA loads (Q tiles, the head's codebook, the value tile) and every
-//                              tcgen05.mma: S = Q.Cp^T, O = W.Vp, S_c = Q.Cc_sel^T, O += W_c.Vc, and the
-//                              denominators Z = W.1 through a one-column "ones" operand.
-//   parent warps (8)           two threads per query row: count-weighted logits t = scale*s + log2 n_j
-//                              (empty parents: -inf), row maximum, p = 2^(t - m), z = sum p  (Eq.
-//                              "vqflashattention": p_ij = A_ij n_j), importance partial sums of p / z
-//                              (Eq. "importance"), bf16 weights written back to TMEM where the value MMA
-//                              reads them as its A operand.
-//   selector (1 warp)          importance -> top-P by bisection on the bit pattern, ties to the lower index
-//                              ("Child spawning"); removes the refined parents from the value tile and from
-//                              the ones operand; gathers the selected parents' child codewords and child
-//                              value rows (Algorithm 2, child loop).
-//   child warps (4)            one thread per row: child logits -> running maximum (rescaling O and Z only
-//                              when it moves by more than 2^8), weights to TMEM; then Y = O / Z.
-//
-// Values enter as per-codeword MEANS (value sum / count, written by the aggregation's finalize kernel) and
-// the counts ride in the weights, so numerator and denominator are plain sums over the same bf16 weights:
-//   Y_i = sum_j p_ij mean_j / sum_j p_ij,   p_ij = n_j exp(s_ij - m_i)      (same value as Eq. "aggregates" form).
-// Every wait is a bounded mbarrier wait; a wait that gives up records a code in the status word, every
-// role leaves its loop, and the CTA frees its TMEM and returns.
+// One CTA = one query tile of 128 rows of one (batch, head) at a time; each row is handled by NQ threads
+// (column slices).  Values enter as per-codeword MEANS with the key counts multiplied into the weights.
+// Flow of a tile:
+//   parents   S = Q . Cp^T                 tcgen05.mma, fp32 accumulator in TMEM columns [0, M)
+//             read once into registers: row maximum over non-empty parents, exp2, exact
+//             denominator z                                         (Eq. "vqflashattention")
+//             importance w_j = n_j sum_i A_ij / z_i from the fp32 weights  (Eq. "importance")
+//             top-P by rank, ties to the lower index                ("Child spawning")
+//             bf16 weights A_ij n_j -> shared memory; a refined parent's row of the value tile is cleared
+//             O = (A n) . mean_p           tcgen05.mma into TMEM columns [CT, CT + d)
+//   children  of the selected parents, in chunks of <= CHW columns: gathered codeword rows,
+//             S_c = Q . Cc_sel^T, running maximum (non-empty children only), O rescaled in TMEM if a
+//             row's maximum moved, bf16 weights, O += A_c . Vbar_c   (Algorithm 2, child loop)
+//   Y = O / z, z accumulated from the same bf16-rounded weights as the numerator.
+// Empty codewords are excluded from every maximum and contribute nothing (their count and value sum
+// are zero; their weight is clamped so that it stays finite) - appendix on numerical stability.
+// The gathers of the first child chunk are issued early so that their latency hides behind the weight
+// conversion and the parents' second MMA.
 #include "avq_tc_common.cuh"
 
 namespace avq {
@@ -32,17 +26,10 @@ namespace {
 using namespace tc;
 
 constexpr int kRows = 128;
-constexpr int kParentWarps = 8;
-// warps 8..11 are the child warps (a warp reaches the TMEM lane quarter warp % 4)
-constexpr int kIssuerWarp = 12;
-constexpr int kSelectWarp = 13;
-constexpr int kLoaderWarp = 14;
-constexpr int kAttendThreads = 15 * 32;
-constexpr float kLazyLog2 = 8.f;        // a child maximum within 2^8 of the running one does not move it
 
 struct AttendParams {
   const __nv_bfloat16* Cc;    // [H, M, C, d]
-  const __nv_bfloat16* Vcb;   // [B*H, M, C, d]  child value means
+  const __nv_bfloat16* Vcb;   // [B*H, M, C, d]
   const float* np_;           // [B*H, M]
   const float* nc;            // [B*H, M, C]
   __nv_bfloat16* Y;           // [B*H, Nq, d]
@@ -56,56 +43,6 @@ struct AttendParams {
   float scale_log2e;
 };
 
-// Barrier indices (one uint64_t each).
-enum Bar : int {
-  B_QFULL = 0,      // [2] query tile landed (per Q buffer)
-  B_CPFULL = 2,     // parent codebook landed
-  B_VPFULL = 3,     // value tile landed
-  B_SFULL = 4,      // [2] S = Q.Cp^T done (per tile parity)
-  B_WREADY = 6,     // [2] parent weights in TMEM (256 arrivals)
-  B_IMP = 8,        // [2] importance partial sums in shared memory (256 arrivals)
-  B_VCLR = 10,      // refined parents removed from the value tile / ones operand (32 arrivals)
-  B_PVDONE = 11,    // O = W.Vp done
-  B_CCREADY = 12,   // [2] child codes and values of a chunk gathered (TMA bytes + one arrival, per slot)
-  B_SCFULL = 14,    // child logits done
-  B_WCREADY = 15,   // child weights in TMEM (128 arrivals)
-  B_CPVDONE = 16,   // [2] O += W_c.Vc done (per slot)
-  B_OFREE = 18,     // output accumulators read (128 arrivals)
-  B_PAIR = 19,      // [4] the two parent warps of a row quarter exchange (64 arrivals)
-  B_PSYNC = 23,     // all parent threads (256 arrivals)
-  B_DRAIN = 24,
-  B_QFREE = 25,     // [2] every MMA that read this Q buffer has completed (issuer -> loader)
-  B_XFREE = 27,     // the value tile's memory may take the next tile's values (issuer -> loader)
-  B_COUNT = 28
-};
-
-template <int D, int CT, int CHW, bool ALIAS>
-struct Smem {
-  static constexpr int kQ = kRows * D * 2;                   // one query tile
-  static constexpr int kCp = CT * D * 2;
-  static constexpr int kX = CT * D * 2;                      // value tile (rows = parents)
-  static constexpr int kSlot = 2 * CHW * D * 2;              // child codes + child values of one chunk
-  static constexpr int kOnesP = (CT / 64) * 2048;
-  static constexpr int kOnesC = (CHW / 64) * 2048;
-  static constexpr int oQ = 0;
-  static constexpr int oCp = oQ + 2 * kQ;
-  static constexpr int oX = oCp + kCp;
-  static constexpr int oSlots = ALIAS ? oX : oX + kX;
-  static constexpr int oOnesP = ALIAS ? oX + kX : oSlots + 2 * kSlot;
-  static constexpr int oOnesC = oOnesP + kOnesP;
-  static constexpr int oLb = oOnesC + kOnesC;                // float [2][CT]
-  static constexpr int oLbc = oLb + 2 * CT * 4;              // float [2][CHW]
-  static constexpr int oWpart = oLbc + 2 * CHW * 4;          // float [2][4][CT]
-  static constexpr int oXm = oWpart + 8 * CT * 4;            // float [2][128]
-  static constexpr int oXz = oXm + 2 * kRows * 4;            // float [2][128]
-  static constexpr int oMrow = oXz + 2 * kRows * 4;          // float [2][128]
-  static constexpr int oSel = oMrow + 2 * kRows * 4;         // int [CT]
-  static constexpr int oBars = oSel + CT * 4;                // uint64 [B_COUNT]
-  static constexpr int oMisc = oBars + B_COUNT * 8;          // tmem slot, abort flag, early exit
-  static constexpr int kTotal = oMisc + 16;
-  static_assert(!ALIAS || 2 * kSlot <= kX, "child slots must fit the value tile");
-};
-
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -115,7 +52,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-__device__ __forceinline__ float max3(float a, float b, float c) { return fmaxf(a, fmaxf(b, c)); }
 
 // Column sums over the 32 lanes of a warp of V values per lane.  Returns, in every lane, the
 // sum of column (lane >> (5 - log2 V)).  V = 32: 31 shuffles instead of 160.
@@ -142,736 +78,674 @@ __device__ __forceinline__ float transpose_reduce(float (&v)[V], int lane) {
   return v[0];
 }
 
-// Walks `ncols` (a multiple of 16) TMEM columns of this thread's lane, starting at `t`, in chunks of 32 and
-// one closing chunk of 16 if needed (a TMEM round trip costs a few hundred cycles: wide chunks amortise it,
-// and the other warps of the scheduler work meanwhile).  The functors get the raw registers and the chunk's
-// first column.
-template <typename F32, typename F16>
-__device__ __forceinline__ void tmem_walk(uint32_t t, int ncols, F32&& f32, F16&& f16) {
-  const int nfull = ncols >> 5;
-  for (int i = 0; i < nfull; ++i) {
-    uint32_t a[32];
-    tmem_ld32_issue(t + (uint32_t)(i * 32), a);
-    tmem_ld_wait32(a);
-    f32(a, i * 32);
-  }
-  if (ncols & 16) {
-    uint32_t tl[16];
-    tmem_ld16_issue(t + (uint32_t)(nfull * 32), tl);
-    tmem_ld_wait16(tl);
-    f16(tl, nfull * 32);
-  }
+// The NQ warps that share a quarter of the rows (warp % 4 == q) exchange per-row values through shared
+// memory; they synchronise among themselves on named barrier q + 1 instead of stalling the whole CTA.
+template <int NQ>
+__device__ __forceinline__ void row_sync(int q) {
+  asm volatile("bar.sync %0, %1;" ::"r"(q + 1), "r"(32 * NQ) : "memory");
 }
-__device__ __forceinline__ float u2f(uint32_t u) { return __uint_as_float(u); }
-__device__ __forceinline__ uint32_t f2u(float f) { return __float_as_uint(f); }
 
-// D: head dimension; CT: parent tile width (>= M); CHW: child chunk width; SB: TMEM buffers for the parent
-// logits (2 where the columns allow it: the next tile's logits are then computed before this tile's value
-// MMA); ALIAS: the child chunk slots live inside the value tile's shared memory (used between a tile's
-// value MMA and the reload of the value tile for the next tile).
-template <int D, int CT, int CHW, int SB, bool ALIAS>
-__global__ void __launch_bounds__(kAttendThreads, 1)
+// Multiplies 16 fp32 weights by their codewords' key counts, rounds the products to bf16, stores them at
+// (row r, columns col0..col0+15) of the K-major swizzled A tile, and returns the sum of the rounded
+// products times a 0/1 mask (`keep16`: 0 for a refined parent, whose value row has been cleared).
+__device__ __forceinline__ float store_weights16(unsigned char* A, int r, int col0, const float* cnt16,
+                                                 const float* keep16, const float (&a)[16]) {
+  const float4* n4 = reinterpret_cast<const float4*>(cnt16);
+  const float4* k4 = reinterpret_cast<const float4*>(keep16);
+  uint32_t pk[8];
+  float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;         // independent partial sums: no 16-deep FMA chain
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const float4 n = n4[u];
+    const float4 k = k4[u];
+    const uint32_t p0 = pack_bf16(a[4 * u] * n.x, a[4 * u + 1] * n.y);
+    const uint32_t p1 = pack_bf16(a[4 * u + 2] * n.z, a[4 * u + 3] * n.w);
+    z0 = fmaf(__uint_as_float(p0 << 16), k.x, z0);
+    z1 = fmaf(__uint_as_float(p0 & 0xFFFF0000u), k.y, z1);
+    z2 = fmaf(__uint_as_float(p1 << 16), k.z, z2);
+    z3 = fmaf(__uint_as_float(p1 & 0xFFFF0000u), k.w, z3);
+    pk[2 * u] = p0;
+    pk[2 * u + 1] = p1;
+  }
+  const float z = (z0 + z1) + (z2 + z3);
+  unsigned char* sub = A + (col0 >> 6) * (kRows * 128);
+  *reinterpret_cast<uint4*>(sub + sw128_offset(r, col0 & 63)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+  *reinterpret_cast<uint4*>(sub + sw128_offset(r, (col0 & 63) + 8)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+  return z;
+}
+
+// NQ = threads per query row: 1, 2 or 4.  Small tiles take NQ = 1 so that four CTAs share an SM and
+// overlap each other's load / MMA / softmax phases; the largest take NQ = 4.
+// CT = parent tile width (64, 128 or 256, >= M), a compile-time constant so that every shared-memory
+// offset folds into the instruction stream instead of occupying a register.
+template <int D, int NQ, int CT>
+__global__ void __launch_bounds__(128 * NQ, 4 / NQ)
 tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmCp,
-                 const __grid_constant__ CUtensorMap tmVpb, const __grid_constant__ CUtensorMap tmCc,
-                 const __grid_constant__ CUtensorMap tmVcb, const AttendParams p) {
+                 const __grid_constant__ CUtensorMap tmVpb, const __grid_constant__ CUtensorMap tmY,
+                 const AttendParams p) {
   // 1024-byte alignment (swizzle atoms) is requested from the launch, not computed from the pointer, so
   // that the compiler keeps every access in the shared address space.
   extern __shared__ __align__(1024) unsigned char smem[];
-  using L = Smem<D, CT, CHW, ALIAS>;
+  constexpr int kThreads = 128 * NQ;
+  constexpr int kScLane = kThreads / 2;                  // lane 0 of a warp in the other half of the CTA
   constexpr int kSubD = D / 64;
-  constexpr int kLogChunks = (D == 128) ? 4 : 3;         // log2 of the 16-byte chunks per codeword row
-  constexpr int kChunks = 1 << kLogChunks;
-  constexpr uint32_t kColS = 0, kColSc = SB * CT, kColO = kColSc + CHW, kColZ = kColO + D;
-  static_assert(kColZ + 16 <= 512, "TMEM columns");
-
-  unsigned char* Qs = smem + L::oQ;
-  unsigned char* Cps = smem + L::oCp;
-  unsigned char* Xs = smem + L::oX;
-  unsigned char* slots = smem + L::oSlots;
-  unsigned char* ones_p = smem + L::oOnesP;
-  unsigned char* ones_c = smem + L::oOnesC;
-  float* lb = reinterpret_cast<float*>(smem + L::oLb);
-  float* lbc = reinterpret_cast<float*>(smem + L::oLbc);
-  float* wpart = reinterpret_cast<float*>(smem + L::oWpart);
-  float* xm = reinterpret_cast<float*>(smem + L::oXm);
-  float* xz = reinterpret_cast<float*>(smem + L::oXz);
-  float* m_row = reinterpret_cast<float*>(smem + L::oMrow);
-  int* sel_list = reinterpret_cast<int*>(smem + L::oSel);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::oBars);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::oMisc);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::oMisc + 4);
-  volatile int* early_exit = reinterpret_cast<volatile int*>(smem + L::oMisc + 8);
+  constexpr int kLogD = (D == 128) ? 7 : 6;
+  constexpr int kLogChunks = kLogD - 3;                  // 16-byte chunks per codeword row
+  constexpr int CHW = CT < 128 ? CT : 128;               // child chunk width
+  constexpr int QW = CT / NQ, QWC = CHW / NQ;
+  constexpr int subA = CT >> 6;                          // 64-column sub-tiles of an A / value tile
+  constexpr int ca_bytes = (CT * D * 2 > subA * kRows * 128) ? CT * D * 2 : subA * kRows * 128;
+  const int M = p.M, C = p.C, P = p.P, logC = p.logC;
+  unsigned char* Qs = smem;                              // kSubD x [128 x 128 B]
+  unsigned char* CA = Qs + kSubD * kRows * 128;          // parent codes, later the bf16 weights
+  unsigned char* Vs = CA + ca_bytes;                     // value rows: kSubD x [rows x 128 B], rows = M or a chunk's children
+  unsigned char* CC = Vs + subA * D * 128;               // kSubD x [CHW x 128 B] gathered child codes
+  float* cnt = reinterpret_cast<float*>(CC + CHW * D * 2);   // [CT] key counts of the parents
+  float* bias = cnt + CT;                                // [CT] 0 for non-empty parents, -inf for empty
+  float* cntk = bias + CT;                               // [CT] 1 for a parent that keeps its own term, 0 once refined
+  float* cntc = cntk + CT;                               // [CHW] key counts of the child chunk
+  float* biasc = cntc + CHW;                             // [CHW]
+  float* keepc = biasc + CHW;                            // [CHW] all ones (children are never removed)
+  float* w = keepc + CHW;                                // [256] importance
+  float* wpart = w + 256;                                // [4][CT]
+  float* xm = wpart + 4 * CT;                            // [NQ][128] exchange between the threads of a row
+  float* xz = xm + NQ * kRows;                           // [NQ][128]
+  float* xz2 = xz + NQ * kRows;                          // [NQ][128]
+  int* sel_list = reinterpret_cast<int*>(xz2 + NQ * kRows);   // [256]
+  uint32_t* wmask = reinterpret_cast<uint32_t*>(sel_list + 256);   // [16]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(wmask + 18);        // [5]  (wmask[16] is a scratch word)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int M = p.M, C = p.C, P = p.P, logC = p.logC;
-  const int PC = P * C;
-  const int nchunks = (PC + CHW - 1) / CHW;
-  const float sc = p.scale_log2e;
-  const bool need_w = (P > 0 && P < M) || p.importance_out != nullptr;
-
-  // This CTA's run of tiles.
-  const int t_begin = (int)(((long long)p.total_tiles * blockIdx.x) / gridDim.x);
-  const int t_end = (int)(((long long)p.total_tiles * (blockIdx.x + 1)) / gridDim.x);
-  const int T = t_end - t_begin;
-
-#define AVQ_WAIT(bar_index, parity) \
-  mbar_wait(&bars[bar_index], (uint32_t)(parity), abort_flag, p.status_word, DEV_TIMEOUT_ATTEND)
-
-  // ------------------------------------------------------------------ set-up
-  auto issue_q = [&](int n) {                            // issuer lane only
-    const int tile = t_begin + n, tb = tile / p.nblk, ti0 = (tile - tb * p.nblk) * kRows;
-    uint64_t* bar = &bars[B_QFULL + (n & 1)];
-    mbar_expect_tx(bar, (uint32_t)L::kQ);
+  const int q = warp & 3, cq = warp >> 2, r = q * 32 + lane;
+  const int colbase = cq * QW;
+  uint64_t* bar_q = &bars[0];                            // query tile landed
+  uint64_t* bar_ld1 = &bars[1];                          // parent value rows landed
+  uint64_t* bar_s = &bars[2];
+  uint64_t* bar_pv = &bars[3];
+  uint64_t* bar_cp = &bars[4];                           // parent codebook landed
+  // A CTA works through the tiles blockIdx.x, blockIdx.x + gridDim.x, ... (the grid is one wave of CTAs).
+  // The next tile's Q is loaded as soon as this tile's last logits are done, its codebook as soon as this
+  // tile's last value MMA is done, so the set-up, the loads and the first MMA of a tile hide behind the tail
+  // of the tile before.  The output is staged where the next tile's first loads do not go: in the child-code
+  // buffer when that is as large as a Q tile (CT >= 128), else across the value tile and the child-code
+  // buffer, which are adjacent and together as large (the next tile's value rows then load a little later).
+  constexpr bool kChain = true;
+  constexpr bool kStageInCC = CT >= 128;
+  static_assert(kStageInCC || (CT * D * 2 + CHW * D * 2 == kSubD * kRows * 128), "staging area");
+  auto issue_q = [&](int t) {                            // thread 0 only
+    const int tb = t / p.nblk, ti0 = (t - tb * p.nblk) * kRows;
+    mbar_expect_tx(bar_q, (uint32_t)(kSubD * kRows * 128));
 #pragma unroll
-    for (int s = 0; s < kSubD; ++s)
-      tma_load_3d(Qs + (n & 1) * L::kQ + s * kRows * 128, &tmQ, s * 64, ti0, tb, bar);
+    for (int s = 0; s < kSubD; ++s) tma_load_3d(Qs + s * kRows * 128, &tmQ, s * 64, ti0, tb, bar_q);
   };
-  auto prefetch_q = [&](int n) {
-    const int tile = t_begin + n, tb = tile / p.nblk, ti0 = (tile - tb * p.nblk) * kRows;
+  auto issue_cp = [&](int t) {
+    const int th = (t / p.nblk) % p.H;
+    mbar_expect_tx(bar_cp, (uint32_t)(kSubD * M * 128));
 #pragma unroll
-    for (int s = 0; s < kSubD; ++s) tma_prefetch_l2_3d(&tmQ, s * 64, ti0, tb);
+    for (int s = 0; s < kSubD; ++s) tma_load_2d(CA + s * M * 128, &tmCp, s * 64, th * M, bar_cp);
   };
-  auto issue_cp = [&](int h) {
-    mbar_expect_tx(&bars[B_CPFULL], (uint32_t)(kSubD * M * 128));
+  auto issue_vp = [&](int t) {
+    const int tb = t / p.nblk;
+    mbar_expect_tx(bar_ld1, (uint32_t)(kSubD * M * 128));
 #pragma unroll
-    for (int s = 0; s < kSubD; ++s) tma_load_2d(Cps + s * M * 128, &tmCp, s * 64, h * M, &bars[B_CPFULL]);
-  };
-  auto issue_vp = [&](int bh) {
-    mbar_expect_tx(&bars[B_VPFULL], (uint32_t)(kSubD * M * 128));
-#pragma unroll
-    for (int s = 0; s < kSubD; ++s) tma_load_2d(Xs + s * M * 128, &tmVpb, s * 64, bh * M, &bars[B_VPFULL]);
+    for (int s = 0; s < kSubD; ++s) tma_load_2d(Vs + s * M * 128, &tmVpb, s * 64, tb * M, bar_ld1);
   };
 
-  if (warp == kIssuerWarp && lane == 0) {
+  __shared__ int early_exit;
+
+  // ---- Part 1 touches only the caller's Q and Cp, so it may run while the kernel that produces the
+  // aggregates is still finishing (programmatic dependent launch): barriers, TMEM, the Q / Cp loads and
+  // S = Q . Cp^T.
+  if (tid == 0) {
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmCp);
     prefetch_tmap(&tmVpb);
-    prefetch_tmap(&tmCc);
-    prefetch_tmap(&tmVcb);
-    auto init = [&](int i, int n, uint32_t count) {
-      for (int u = 0; u < n; ++u) mbar_init(&bars[i + u], count);
-    };
-    init(B_QFULL, 2, 1);
-    init(B_CPFULL, 1, 1);
-    init(B_VPFULL, 1, 1);
-    init(B_SFULL, 2, 1);
-    init(B_WREADY, 2, 32 * kParentWarps);
-    init(B_IMP, 2, 32 * kParentWarps);
-    init(B_VCLR, 1, 32);
-    init(B_PVDONE, 1, 1);
-    init(B_CCREADY, 2, 1);
-    init(B_SCFULL, 1, 1);
-    init(B_WCREADY, 1, 128);
-    init(B_CPVDONE, 2, 1);
-    init(B_OFREE, 1, 128);
-    init(B_PAIR, 4, 64);
-    init(B_PSYNC, 1, 32 * kParentWarps);
-    init(B_DRAIN, 1, 1);
-    init(B_QFREE, 2, 1);
-    init(B_XFREE, 1, 1);
+    mbar_init(bar_q, 1);
+    mbar_init(bar_cp, 1);
+    mbar_init(bar_ld1, 1);
+    mbar_init(bar_s, 1);
+    mbar_init(bar_pv, 1);
     mbar_fence_init();
     *abort_flag = 0;
-    *early_exit = 0;
-    // Q and the codebook are the caller's: their loads may go out while the kernel that produces the
-    // aggregates is still finishing (programmatic dependent launch).
-    issue_q(0);
-    if (T > 1) issue_q(1);
-    if (T > 2) prefetch_q(2);
-    issue_cp(((t_begin / p.nblk)) % p.H);
+    issue_q(blockIdx.x);
+    issue_cp(blockIdx.x);
   }
-  if (warp == kSelectWarp) {
+  if (warp == 1) {                                   // not the warp whose lane 0 is busy issuing the loads
     tmem_alloc(tmem_slot, p.tmem_cols);
     tmem_relinquish();
   }
-  // Constant operands: the ones tiles are [16 rows x 64 k] K-major swizzled sub-tiles, row 0 carries the
-  // ones (the other 15 output columns of the denominator MMA stay zero and are never read).
-  for (int u = tid; u < (L::kOnesP + L::kOnesC) / 16; u += kAttendThreads)
-    reinterpret_cast<uint4*>(ones_p)[u] = make_uint4(0u, 0u, 0u, 0u);
-  __syncthreads();
-  for (int u = tid; u < (CHW / 64) * 8; u += kAttendThreads)      // row 0 of every child sub-tile: 128 bytes of 1.0
-    *reinterpret_cast<uint4*>(ones_c + (u >> 3) * 2048 + (u & 7) * 16) =
-        make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
-  fence_proxy_async();
-  pdl_wait();          // from here on the aggregates of this call may be read
-  if (tid == 0)
-    *early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-
-  if (*early_exit) {
-    // a wait expired in an earlier kernel of this call: let the loads already in flight land, then leave
-    if (warp == kIssuerWarp && lane == 0) {
-      AVQ_WAIT(B_QFULL, 0);
-      if (T > 1) AVQ_WAIT(B_QFULL + 1, 0);
-      AVQ_WAIT(B_CPFULL, 0);
-    }
-  } else if (warp == kIssuerWarp) {
-    // ================================================================ issuer
-    if (lane == 0) {
-      const uint32_t idesc_o = umma_idesc_bf16(kRows, D) | (1u << 16);   // B (value rows) is MN-major
-      const uint32_t idesc_z = umma_idesc_bf16(kRows, 16);
-      const uint32_t idesc_s = umma_idesc_bf16(kRows, M);
-      const uint32_t cps = smem_u32(Cps), xs = smem_u32(Xs), onesp = smem_u32(ones_p), onesc = smem_u32(ones_c);
-      uint32_t ph_q[2] = {0, 0}, ph_cp = 0, ph_vclr = 0, ph_pv = 0, ph_cc[2] = {0, 0}, ph_wc = 0,
-               ph_cpv[2] = {0, 0}, ph_of = 0;
-      int g = 0;                                           // child chunks issued so far (slot = g & 1)
-      bool ok = true;
-      auto mma_s = [&](int n) {
-        const uint32_t qa = smem_u32(Qs + (n & 1) * L::kQ);
-        const uint32_t d = tmem_base + kColS + (uint32_t)((n % SB) * CT);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k)
-          umma_bf16(d, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
-                    umma_desc_sw128(cps + (k / 4) * M * 128 + (k % 4) * 32), idesc_s, k > 0);
-        umma_commit(&bars[B_SFULL + (n & 1)]);
-      };
-      ok = AVQ_WAIT(B_QFULL, ph_q[0]) && AVQ_WAIT(B_CPFULL, ph_cp);
-      ph_q[0] ^= 1;
-      ph_cp ^= 1;
-      if (ok) {
-        tc_fence_after();
-        mma_s(0);
-      }
-      for (int n = 0; ok && n < T; ++n) {
-        const int tile = t_begin + n, bh = tile / p.nblk;
-        const bool has_next = n + 1 < T;
-        const int bh_next = (tile + 1) / p.nblk;
-        auto next_logits = [&]() -> bool {                 // S(n+1): codebook of its head, its Q tile
-          if ((bh_next % p.H) != (bh % p.H)) {
-            // the logits MMA of tile n is the last reader of the resident codebook
-            if (!AVQ_WAIT(B_SFULL + (n & 1), (n >> 1) & 1)) return false;
-            issue_cp(bh_next % p.H);
-            if (!AVQ_WAIT(B_CPFULL, ph_cp)) return false;
-            ph_cp ^= 1;
-          }
-          if (!AVQ_WAIT(B_QFULL + ((n + 1) & 1), ph_q[(n + 1) & 1])) return false;
-          ph_q[(n + 1) & 1] ^= 1;
-          tc_fence_after();
-          mma_s(n + 1);
-          return true;
-        };
-        // With two logit buffers the next tile's logits go first: its buffer was released by the value
-        // MMA of tile n-1, and every MMA that read the codebook has completed (waited for below).
-        if (SB == 2 && has_next && !(ok = next_logits())) break;
-
-        // ---- O = W.Vp, Z = W.1   (parents)
-        ok = AVQ_WAIT(B_WREADY + (n & 1), (n >> 1) & 1) && AVQ_WAIT(B_VCLR, ph_vclr);
-        ph_vclr ^= 1;
-        if (ok && n > 0) {
-          ok = AVQ_WAIT(B_OFREE, ph_of);
-          ph_of ^= 1;
-        }
-        if (!ok) break;
-        tc_fence_after();
-        {
-          const uint32_t wbase = tmem_base + kColS + (uint32_t)((n % SB) * CT);
-          const int half_steps = M / 32;                   // K steps (16 parents) per column half
-          // descriptors advance by adding to their 14-bit address field (units of 16 bytes; shared memory
-          // addresses stay below 2^18, so the field cannot carry into the next one)
-          const uint64_t dv = umma_desc_sw128_mn(xs, (uint32_t)(M * 128)), dz = umma_desc_sw128(onesp);
-#pragma unroll 4
-          for (int k = 0; k < M / 16; ++k) {
-            const uint32_t a = wbase + (uint32_t)(k < half_steps ? k * 8 : M / 2 + (k - half_steps) * 8);
-            umma_bf16_ts(tmem_base + kColO, a, dv + (uint64_t)(k * 128), idesc_o, k > 0);
-            umma_bf16_ts(tmem_base + kColZ, a, dz + (uint64_t)((k >> 2) * 128 + (k & 3) * 2), idesc_z, k > 0);
-          }
-          umma_commit(&bars[B_PVDONE]);
-        }
-        // The value MMA must be complete before the value tile is reloaded, before the logit buffer it
-        // read its weights from is overwritten, and (no children) before the Q buffer is reused.
-        ok = AVQ_WAIT(B_PVDONE, ph_pv);
-        ph_pv ^= 1;
-        if (!ok) break;
-        if (!ALIAS && has_next) mbar_arrive(&bars[B_XFREE]);
-        if (SB == 1 && has_next && !(ok = next_logits())) break;
-
-        // ---- children of tile n
-        const uint32_t qa = smem_u32(Qs + (n & 1) * L::kQ);
-        for (int k = 0; ok && k < nchunks; ++k, ++g) {
-          const int slot = g & 1;
-          const int ncols = min(PC - k * CHW, CHW), np16 = (ncols + 15) & ~15;
-          const uint32_t cc = smem_u32(slots + slot * L::kSlot), vc = cc + CHW * D * 2;
-          ok = AVQ_WAIT(B_CCREADY + slot, ph_cc[slot]);
-          ph_cc[slot] ^= 1;
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t idesc_c = umma_idesc_bf16(kRows, np16);
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk)
-            umma_bf16(tmem_base + kColSc, umma_desc_sw128(qa + (kk / 4) * kRows * 128 + (kk % 4) * 32),
-                      umma_desc_sw128(cc + (kk / 4) * np16 * 128 + (kk % 4) * 32), idesc_c, kk > 0);
-          umma_commit(&bars[B_SCFULL]);
-          ok = AVQ_WAIT(B_WCREADY, ph_wc);
-          ph_wc ^= 1;
-          if (!ok) break;
-          tc_fence_after();
-          const uint64_t dvc = umma_desc_sw128_mn(vc, (uint32_t)(np16 * 128)), dzc = umma_desc_sw128(onesc);
-#pragma unroll 4
-          for (int kk = 0; kk < np16 / 16; ++kk) {
-            const uint32_t a = tmem_base + kColSc + (uint32_t)(kk * 8);
-            umma_bf16_ts(tmem_base + kColO, a, dvc + (uint64_t)(kk * 128), idesc_o, true);
-            umma_bf16_ts(tmem_base + kColZ, a, dzc + (uint64_t)((kk >> 2) * 128 + (kk & 3) * 2), idesc_z, true);
-          }
-          umma_commit(&bars[B_CPVDONE + slot]);
-          // the child weights alias the child logits: the next chunk's logits wait for this MMA
-          ok = AVQ_WAIT(B_CPVDONE + slot, ph_cpv[slot]);
-          ph_cpv[slot] ^= 1;
-        }
-        if (!ok) break;
-        if (ALIAS && has_next) mbar_arrive(&bars[B_XFREE]);   // the child slots inside the value tile are free again
-        if (n + 2 < T) mbar_arrive(&bars[B_QFREE + (n & 1)]);  // every MMA that read Q(n) has completed
-      }
-      // every MMA issued above has completed on the normal path; after a failed wait give the ones in
-      // flight (and the loads) time to finish before the CTA's shared memory and TMEM are released
-      umma_commit(&bars[B_DRAIN]);
-      mbar_wait(&bars[B_DRAIN], 0, abort_flag, nullptr, 0);
-      if (*abort_flag) {
-        const unsigned long long t0 = global_timer_ns();
-        while (global_timer_ns() - t0 < 100000ull) { }
-      }
-    }
-  } else if (warp == kLoaderWarp) {
-    // ================================================================ loader: the Q tiles and the value tiles
-    // (a TMA issue costs its thread several hundred cycles, which the MMA issuer cannot spare)
-    if (lane == 0) {
-      issue_vp(t_begin / p.nblk);
-      uint32_t ph_qf[2] = {0, 0}, ph_xf = 0;
-      bool ok = true;
-      for (int n = 0; ok && n < T; ++n) {
-        if (n + 1 < T) {
-          ok = AVQ_WAIT(B_XFREE, ph_xf);
-          ph_xf ^= 1;
-          if (!ok) break;
-          issue_vp((t_begin + n + 1) / p.nblk);
-        }
-        if (n + 2 < T) {
-          ok = AVQ_WAIT(B_QFREE + (n & 1), ph_qf[n & 1]);
-          ph_qf[n & 1] ^= 1;
-          if (!ok) break;
-          issue_q(n + 2);
-          if (n + 3 < T) prefetch_q(n + 3);
-        }
-      }
-    }
-  } else if (warp < kParentWarps) {
-    // ================================================================ parent warps
-    const int q = warp & 3, hf = warp >> 2, r = q * 32 + lane;
-    const int Mh = M >> 1;                                // columns per thread (multiple of 16)
-    const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
-    uint32_t ph_pair = 0, ph_psync = 0;
-    int prev_bh = -1, lsel = 1;
-    auto pair_sync = [&]() -> bool {
-      mbar_arrive(&bars[B_PAIR + q]);
-      const bool ok = AVQ_WAIT(B_PAIR + q, ph_pair);
-      ph_pair ^= 1;
-      return ok;
-    };
-    for (int n = 0; n < T; ++n) {
-      const int tile = t_begin + n, bh = tile / p.nblk, blk = tile - bh * p.nblk;
-      const int rows_valid = min(kRows, p.Nq - blk * kRows);
-      if (bh != prev_bh) {
-        // log2 of the parents' key counts (-inf for an empty parent and for the padding columns): added to the
-        // scaled logit it puts the count into the weight and keeps empty parents out of the maximum
-        lsel ^= 1;
-        for (int j = tid; j < CT; j += 32 * kParentWarps)
-          lb[lsel * CT + j] = j < M ? log2f(p.np_[(size_t)bh * M + j]) : -INFINITY;
-        mbar_arrive(&bars[B_PSYNC]);
-        const bool ok = AVQ_WAIT(B_PSYNC, ph_psync);
-        ph_psync ^= 1;
-        if (!ok) break;
-        prev_bh = bh;
-      }
-      const float* lbt = lb + lsel * CT + hf * Mh;
-      const uint32_t t_s = t_lane + kColS + (uint32_t)((n % SB) * CT + hf * Mh);
-      if (!AVQ_WAIT(B_SFULL + (n & 1), (n >> 1) & 1)) break;
+  const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+  const uint32_t t_s = t_row + (uint32_t)colbase;
+  const uint32_t t_sc = t_row + (uint32_t)(cq * QWC);
+  const uint32_t t_o = t_row + (uint32_t)(CT + cq * (D / NQ));
+  const uint32_t idesc_o = umma_idesc_bf16(kRows, D) | (1u << 16);   // B (the value rows) is MN-major
+  const float sc = p.scale_log2e;
+  uint32_t ph_s = 0, ph_pv = 0, ph_in = 0;               // ph_in: parity of the three load barriers (once per tile)
+  const int PC = P * C;
+  const int my_cols = min(max(M - colbase, 0), QW);      // multiple of 16 (M % 32 == 0, QW % 16 == 0)
+  bool first = true;
+  bool store_pending = false;                            // thread 0: a TMA store may still be reading CC
+  for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+  const int bh = tile / p.nblk, blk = tile - bh * p.nblk, h = bh % p.H;
+  const int i0 = blk * kRows;
+  const int rows_valid = min(kRows, p.Nq - i0);
+  const int next_tile = tile + gridDim.x;
+  const bool has_next = kChain && next_tile < p.total_tiles;
+  if (tid == 0) {
+    const bool q_ok = mbar_wait(bar_q, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+    const bool c_ok = mbar_wait(bar_cp, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+    if (q_ok && c_ok) {
       tc_fence_after();
-
-      // ---- pass 0: t = scale * s + log2 n_j, row maximum; t replaces s in TMEM
-      float mx0 = -INFINITY, mx1 = -INFINITY;
-      auto pass0 = [&](auto& rg, int c0) __attribute__((always_inline)) {
-        constexpr int W = sizeof(rg) / 4;
-        const float4* l4 = reinterpret_cast<const float4*>(lbt + c0);
+      const uint32_t idesc = umma_idesc_bf16(kRows, M);
+      const uint32_t qa = smem_u32(Qs), ca = smem_u32(CA);
 #pragma unroll
-        for (int u = 0; u < W / 4; ++u) {
-          const float4 l = l4[u];
-          const float t0 = fmaf(u2f(rg[4 * u]), sc, l.x), t1 = fmaf(u2f(rg[4 * u + 1]), sc, l.y);
-          const float t2 = fmaf(u2f(rg[4 * u + 2]), sc, l.z), t3 = fmaf(u2f(rg[4 * u + 3]), sc, l.w);
-          mx0 = max3(mx0, t0, t1);
-          mx1 = max3(mx1, t2, t3);
-          rg[4 * u] = f2u(t0); rg[4 * u + 1] = f2u(t1); rg[4 * u + 2] = f2u(t2); rg[4 * u + 3] = f2u(t3);
-        }
-        if constexpr (W == 32) tmem_st32(t_s + (uint32_t)c0, rg);
-        else tmem_st16u(t_s + (uint32_t)c0, rg);
-      };
-      tmem_walk(t_s, Mh, pass0, pass0);
-      tmem_st_wait();
-      xm[hf * kRows + r] = fmaxf(mx0, mx1);
-      if (!pair_sync()) break;
-      const float m = fmaxf(xm[r], xm[kRows + r]);         // finite: at least one parent holds a key
-
-      // ---- pass 1: p = 2^(t - m) (exactly 0 for empty parents), z = sum p; p replaces t in TMEM
-      float z0 = 0.f, z1 = 0.f;
-      auto pass1 = [&](auto& rg, int c0) __attribute__((always_inline)) {
-        constexpr int W = sizeof(rg) / 4;
-#pragma unroll
-        for (int u = 0; u < W; u += 2) {
-          const float e0 = ex2(u2f(rg[u]) - m), e1 = ex2(u2f(rg[u + 1]) - m);
-          z0 += e0;
-          z1 += e1;
-          rg[u] = f2u(e0); rg[u + 1] = f2u(e1);
-        }
-        if constexpr (W == 32) tmem_st32(t_s + (uint32_t)c0, rg);
-        else tmem_st16u(t_s + (uint32_t)c0, rg);
-      };
-      tmem_walk(t_s, Mh, pass1, pass1);
-      tmem_st_wait();
-      xz[hf * kRows + r] = z0 + z1;
-      if (!pair_sync()) break;
-      const float z = xz[r] + xz[kRows + r];
-      if (hf == 0) m_row[(n & 1) * kRows + r] = m;
-
-      // ---- pass 2, one read of p: bf16 weights, packed two per column over this thread's own (already
-      // consumed) columns [hf * Mh, hf * Mh + Mh / 2) - the A operand of the value MMA - and the importance
-      // partial sums: column sums of p_ij / z_i over the tile's valid rows (32 per warp; the selector adds
-      // the four row quarters)                                       (Eq. "importance")
-      const float inv = (r < rows_valid) ? 1.f / z : 0.f;
-      float* wp = wpart + ((n & 1) * 4 + q) * CT + hf * Mh;
-      auto pass2 = [&](auto& rg, int c0) __attribute__((always_inline)) {
-        constexpr int W = sizeof(rg) / 4;
-        uint32_t pk[W / 2];
-#pragma unroll
-        for (int u = 0; u < W / 2; ++u) pk[u] = pack_bf16(u2f(rg[2 * u]), u2f(rg[2 * u + 1]));
-        if constexpr (W == 32) tmem_st16u(t_s + (uint32_t)(c0 >> 1), pk);
-        else tmem_st8(t_s + (uint32_t)(c0 >> 1), pk);
-        if (need_w) {
-          float (&v)[W] = reinterpret_cast<float (&)[W]>(rg);   // in place: the registers are dead after this
-#pragma unroll
-          for (int e = 0; e < W; ++e) v[e] *= inv;
-          const float colsum = transpose_reduce<W>(v, lane);
-          if constexpr (W == 32) wp[c0 + lane] = colsum;
-          else if ((lane & 1) == 0) wp[c0 + (lane >> 1)] = colsum;
-        }
-      };
-      tmem_walk(t_s, Mh, pass2, pass2);
-      mbar_arrive(&bars[B_IMP + (n & 1)]);
-      tmem_st_wait();
-      tc_fence_before();
-      mbar_arrive(&bars[B_WREADY + (n & 1)]);
+      for (int k = 0; k < D / 16; ++k)
+        umma_bf16(tmem_base, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
+                  umma_desc_sw128(ca + (k / 4) * M * 128 + (k % 4) * 32), idesc, k > 0);
     }
-  } else if (warp == kSelectWarp) {
-    // ================================================================ selector
-    constexpr int NI = CT / 32;                            // parents per lane (j = lane + 32 i)
-    uint32_t ph_vp = 0, ph_pv = 0;
-    int g = 0;
-    bool ok = true;
-    for (int n = 0; ok && n < T; ++n) {
-      const int tile = t_begin + n, bh = tile / p.nblk, blk = tile - bh * p.nblk, h = bh % p.H;
-      if (!AVQ_WAIT(B_IMP + (n & 1), (n >> 1) & 1)) break;
-      uint32_t key[NI];
-#pragma unroll
-      for (int i = 0; i < NI; ++i) {
-        const int j = lane + 32 * i;
-        float w = 0.f;
-        if (need_w && j < M) {
-          const float* wp = wpart + (n & 1) * 4 * CT + j;
-          w = (wp[0] + wp[CT]) + (wp[2 * CT] + wp[3 * CT]);
-          if (p.importance_out) p.importance_out[((size_t)bh * p.nblk + blk) * M + j] = w;
-        }
-        key[i] = __float_as_uint(w);                       // non-negative floats order like their bit patterns
-      }
-      // ---- the P largest importances.  T climbs bit by bit to the largest value that at least P keys
-      // reach; the search stops early when exactly P keys reach the candidate.  Keys equal to the final T
-      // fill the remaining places in ascending index order (ties to the lower index).
-      int n_sel = 0;
-      if (P > 0) {
-        uint32_t thr = 0;
-        bool exact = P >= M;                               // P = M: every parent (threshold 0, all keys reach it)
-        if (!exact) {
-          // every lane forms the same count from ballots (no cross-lane reduction on the dependent path)
-          for (int bit = 30; bit >= 0; --bit) {
-            const uint32_t cand = thr | (1u << bit);
-            int c = 0;
-#pragma unroll
-            for (int i = 0; i < NI; ++i) c += __popc(__ballot_sync(0xffffffffu, key[i] >= cand));
-            if (c >= P) {
-              thr = cand;
-              if (c == P) { exact = true; break; }
-            }
-          }
-        }
-        int need = 0;
-        if (!exact) {
-          int c = 0;
-#pragma unroll
-          for (int i = 0; i < NI; ++i) c += __popc(__ballot_sync(0xffffffffu, key[i] > thr));
-          need = P - c;                                    // places left for keys equal to the threshold
-        }
-#pragma unroll
-        for (int i = 0; i < NI; ++i) {
-          const int j = lane + 32 * i;
-          const bool valid = j < M;
-          uint32_t m_sel = __ballot_sync(0xffffffffu, valid && (exact ? key[i] >= thr : key[i] > thr));
-          if (!exact) {
-            uint32_t m_eq = __ballot_sync(0xffffffffu, valid && key[i] == thr);
-            const int have = __popc(m_eq);
-            if (have > need) {                              // keep the `need` lowest lanes of this group
-              const uint32_t pos = need > 0 ? __fns(m_eq, 0, need + 1) : (uint32_t)__ffs(m_eq) - 1u;
-              m_eq &= (pos >= 32u) ? 0xffffffffu : ((1u << pos) - 1u);
-            }
-            need -= __popc(m_eq);
-            m_sel |= m_eq;
-          }
-          if (m_sel & (1u << lane)) {
-            const int pos = n_sel + __popc(m_sel & ((1u << lane) - 1u));
-            sel_list[pos] = j;
-            if (p.topp_out) p.topp_out[((size_t)bh * p.nblk + blk) * P + pos] = j;
-          }
-          n_sel += __popc(m_sel);
-        }
-      }
-      __syncwarp();
+    umma_commit(bar_s);
+    if (!kStageInCC && !first) {
+      // the value tile was the staging area of the tile before: reload it once that store has read it
+      tma_store_wait_read();
+      store_pending = false;
+      issue_vp(tile);
+    }
+  }
 
-      // ---- the value tile of this tile has landed: remove the refined parents from it and from the ones
-      // operand (row 0 of the ones tile is rewritten first: the tile before cleared other entries)
-      if (!AVQ_WAIT(B_VPFULL, ph_vp)) break;
-      ph_vp ^= 1;
-      if (lane * 8 < CT) {
-        uint32_t one[4];
+  // ---- Part 2 reads what the earlier kernels of this call wrote: status word, counts, value sums.
+  if (first) {
+    pdl_wait();
+    if (tid == 0) {
+      // a wait that expired in an earlier CTA or kernel of this call: do not start more work
+      early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
+      issue_vp(tile);
+    }
+  }
+  for (int j = tid; j < CT; j += kThreads) {
+    const float n = j < M ? p.np_[(size_t)bh * M + j] : 0.f;
+    cnt[j] = n;
+    bias[j] = n > 0.f ? 0.f : -INFINITY;
+    cntk[j] = 1.f;
+  }
+  __syncthreads();
+  if (first && early_exit) {
+    // let the MMA and the load already in flight finish, then leave cleanly
+    mbar_wait(bar_s, 0, abort_flag, nullptr, 0);
+    mbar_wait(bar_ld1, 0, abort_flag, nullptr, 0);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
+    return;
+  }
+  first = false;
+
+  // ---- parents: row maximum over non-empty codewords (empty ones carry a -inf bias)
+  mbar_wait(bar_s, ph_s, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+  ph_s ^= 1;
+  tc_fence_after();
+  if (tid == 0 && has_next && PC == 0) issue_q(next_tile);   // no child logits will read this Q tile
+  // This thread's QW (<= 64) parent logits are read from TMEM once and stay in registers through the
+  // maximum, the exponentials, the importance sums and the conversion to bf16.
+  float a[QW];
+  float mx = -INFINITY, mx2 = -INFINITY;
+#pragma unroll
+  for (int c0 = 0; c0 < QW; c0 += 16) {
+    if (c0 < my_cols) {                                  // warp-uniform
+      float s[16];
+      tmem_ld16(t_s + c0, s);
+      const float4* b4 = reinterpret_cast<const float4*>(bias + colbase + c0);
+      // the biased logit stays in the register: an empty parent's -inf becomes a weight of exactly 0
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float4 b = b4[u];
+        a[c0 + 4 * u] = s[4 * u] + b.x;
+        a[c0 + 4 * u + 1] = s[4 * u + 1] + b.y;
+        a[c0 + 4 * u + 2] = s[4 * u + 2] + b.z;
+        a[c0 + 4 * u + 3] = s[4 * u + 3] + b.w;
+        mx = fmaxf(mx, fmaxf(a[c0 + 4 * u], a[c0 + 4 * u + 1]));
+        mx2 = fmaxf(mx2, fmaxf(a[c0 + 4 * u + 2], a[c0 + 4 * u + 3]));
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 16; ++e) a[c0 + e] = 0.f;
+    }
+  }
+  float m_run = fmaxf(mx, mx2) * sc;                    // scale > 0: the maximum commutes with it
+  if (NQ > 1) {
+    xm[cq * kRows + r] = m_run;
+    row_sync<NQ>(q);
+#pragma unroll
+    for (int u = 0; u < NQ; ++u) m_run = fmaxf(m_run, xm[u * kRows + r]);
+  }
+  // m_run is finite: at least one parent holds a key.
+
+  // ---- fp32 weights; exact denominator of the parent pass.  Empty parents carry a logit of -inf, hence
+  // a weight of exactly zero; every other logit is at most the maximum (up to one rounding).
+  float zfull = 0.f;
+  {
+    float zf0 = 0.f, zf1 = 0.f, zf2 = 0.f, zf3 = 0.f;
+    const float negm = -m_run;
+#pragma unroll
+    for (int c0 = 0; c0 < QW; c0 += 16) {
+      if (c0 < my_cols) {
+        const float4* n4 = reinterpret_cast<const float4*>(cnt + colbase + c0);
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          const int j = lane * 8 + 2 * u;
-          one[u] = (j < M ? 0x3F80u : 0u) | (j + 1 < M ? 0x3F800000u : 0u);
-        }
-        *reinterpret_cast<uint4*>(ones_p + ((lane * 8) >> 6) * 2048 + ((lane * 8) & 63) * 2) =
-            make_uint4(one[0], one[1], one[2], one[3]);
-      }
-      __syncwarp();
-      for (int u = lane; u < n_sel; u += 32) {
-        const int j = sel_list[u];
-        *reinterpret_cast<unsigned short*>(ones_p + (j >> 6) * 2048 + (j & 63) * 2) = 0;
-      }
-      for (int u = lane; u < (n_sel << kLogChunks); u += 32) {
-        const int row = sel_list[u >> kLogChunks], ch = u & (kChunks - 1);
-        *reinterpret_cast<uint4*>(Xs + (ch >> 3) * (M * 128) + sw128_offset(row, (ch & 7) * 8)) =
-            make_uint4(0u, 0u, 0u, 0u);
-      }
-      fence_proxy_async();
-      mbar_arrive(&bars[B_VCLR]);
-
-      // ---- child chunks of this tile: codeword rows and value-mean rows of the selected parents' children
-      if (nchunks > 0 && ALIAS) {
-        // the slots lie inside the value tile: wait until this tile's value MMA has read it
-        if (!AVQ_WAIT(B_PVDONE, ph_pv)) break;
-        ph_pv ^= 1;
-      }
-      const __nv_bfloat16* Cch = p.Cc + (size_t)h * M * C * D;
-      const __nv_bfloat16* Vch = p.Vcb + (size_t)bh * M * C * D;
-      const float* ncb = p.nc + (size_t)bh * M * C;
-      for (int k = 0; k < nchunks; ++k, ++g) {
-        const int slot = g & 1;
-        if (g >= 2) {                                      // the chunk that used this slot before must be consumed
-          if (!(ok = AVQ_WAIT(B_CPVDONE + slot, ((g >> 1) - 1) & 1))) break;
-        }
-        const int e_first = k * CHW;
-        const int ncols = min(PC - e_first, CHW), np16 = (ncols + 15) & ~15;
-        unsigned char* cc = slots + slot * L::kSlot;
-        unsigned char* vc = cc + CHW * D * 2;
-        float* lbs = lbc + slot * CHW;
-        for (int i = lane; i < CHW; i += 32) {
-          float l = -INFINITY;
-          if (i < ncols) {
-            const int e = e_first + i;
-            l = log2f(__ldg(ncb + ((size_t)sel_list[e >> logC] << logC) + (e & (C - 1))));
-          }
-          lbs[i] = l;
-        }
-        // Rows of the chunk as K-major / row-per-codeword tiles of np16 rows (sub-tiles of 64 columns).  The
-        // C children of a selected parent are C consecutive rows in global memory and in the tile: one TMA box
-        // per (parent, sub-tile) for the codes and one for the value means, a lane per parent.  Padding rows
-        // (a chunk that ends off a multiple of 16) are zeroed by hand.
-        const int npar = ncols >> logC;                    // selected parents in this chunk
-        const int p_first = e_first >> logC;
-        uint64_t* bar = &bars[B_CCREADY + slot];
-        if (np16 > ncols) {
-          for (int u = lane; u < ((np16 - ncols) << kLogChunks); u += 32) {
-            const int row = ncols + (u >> kLogChunks), ch = u & (kChunks - 1);
-            const uint32_t off = (uint32_t)((ch >> 3) * (np16 * 128)) + sw128_offset(row, (ch & 7) * 8);
-            *reinterpret_cast<uint4*>(cc + off) = make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4*>(vc + off) = make_uint4(0u, 0u, 0u, 0u);
-          }
-          fence_proxy_async();
-        }
-        __syncwarp();
-        if (lane == 0) mbar_expect_tx(bar, (uint32_t)(ncols * D * 2 * 2));   // the one arrival + all the bytes
-        __syncwarp();
-        for (int i = lane; i < npar; i += 32) {
-          const int par = sel_list[p_first + i];
-          const int row_c = (h * M + par) << logC, row_v = (bh * M + par) << logC;
-#pragma unroll
-          for (int sd = 0; sd < kSubD; ++sd) {
-            const uint32_t off = (uint32_t)(sd * (np16 * 128) + ((i << logC) * 128));
-            tma_load_2d(cc + off, &tmCc, sd * 64, row_c, bar);
-            tma_load_2d(vc + off, &tmVcb, sd * 64, row_v, bar);
-          }
+          const float4 n = n4[u];
+          a[c0 + 4 * u] = ex2(fmaf(a[c0 + 4 * u], sc, negm));
+          a[c0 + 4 * u + 1] = ex2(fmaf(a[c0 + 4 * u + 1], sc, negm));
+          a[c0 + 4 * u + 2] = ex2(fmaf(a[c0 + 4 * u + 2], sc, negm));
+          a[c0 + 4 * u + 3] = ex2(fmaf(a[c0 + 4 * u + 3], sc, negm));
+          zf0 = fmaf(a[c0 + 4 * u], n.x, zf0);
+          zf1 = fmaf(a[c0 + 4 * u + 1], n.y, zf1);
+          zf2 = fmaf(a[c0 + 4 * u + 2], n.z, zf2);
+          zf3 = fmaf(a[c0 + 4 * u + 3], n.w, zf3);
         }
       }
     }
-    cp_async_wait_all();
-  } else {
-    // ================================================================ child warps
-    const int q = warp & 3, r = q * 32 + lane;
-    const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
-    const uint32_t t_sc = t_lane + kColSc, t_o = t_lane + kColO, t_z = t_lane + kColZ;
-    uint32_t ph_sc = 0, ph_pv = 0;
-    int g = 0;
-    bool ok = true;
-    for (int n = 0; ok && n < T; ++n) {
-      const int tile = t_begin + n, bh = tile / p.nblk, blk = tile - bh * p.nblk;
-      const int i0 = blk * kRows;
-      const int rows_valid = min(kRows, p.Nq - i0);
-      if (nchunks == 0) {
-        ok = AVQ_WAIT(B_PVDONE, ph_pv);
-        ph_pv ^= 1;
-        if (!ok) break;
-        tc_fence_after();
-      }
-      float m_run = 0.f;
-      for (int k = 0; k < nchunks; ++k, ++g) {
-        const int slot = g & 1;
-        const int ncols = min(PC - k * CHW, CHW), np16 = (ncols + 15) & ~15;
-        // the logits of this chunk are done; so is every MMA issued before them (the parents' value MMA,
-        // the chunk before): O and Z may be rescaled
-        ok = AVQ_WAIT(B_SCFULL, ph_sc);
-        ph_sc ^= 1;
-        if (!ok) break;
-        tc_fence_after();
-        if (k == 0) m_run = m_row[(n & 1) * kRows + r];
-        const float* lbs = lbc + slot * CHW;
-        float mx0 = -INFINITY, mx1 = -INFINITY;
-        auto cpass0 = [&](auto& rg, int c0) __attribute__((always_inline)) {
-          constexpr int W = sizeof(rg) / 4;
-          const float4* l4 = reinterpret_cast<const float4*>(lbs + c0);
+    zfull = (zf0 + zf1) + (zf2 + zf3);
+    if (NQ > 1) {
+      xz[cq * kRows + r] = zfull;
+      row_sync<NQ>(q);
+      zfull = 0.f;
 #pragma unroll
-          for (int u = 0; u < W / 4; ++u) {
-            const float4 l = l4[u];
-            const float t0 = fmaf(u2f(rg[4 * u]), sc, l.x), t1 = fmaf(u2f(rg[4 * u + 1]), sc, l.y);
-            const float t2 = fmaf(u2f(rg[4 * u + 2]), sc, l.z), t3 = fmaf(u2f(rg[4 * u + 3]), sc, l.w);
-            mx0 = max3(mx0, t0, t1);
-            mx1 = max3(mx1, t2, t3);
-            rg[4 * u] = f2u(t0); rg[4 * u + 1] = f2u(t1); rg[4 * u + 2] = f2u(t2); rg[4 * u + 3] = f2u(t3);
-          }
-          if constexpr (W == 32) tmem_st32(t_sc + (uint32_t)c0, rg);
-          else tmem_st16u(t_sc + (uint32_t)c0, rg);
-        };
-        tmem_walk(t_sc, np16, cpass0, cpass0);
-        tmem_st_wait();
-        // Any reference value works as long as numerator and denominator share it.  The running one is kept
-        // unless the children exceed it by more than 2^kLazyLog2 (weights up to that factor above 1 are
-        // harmless in fp32 and bf16), which spares most rows the rescaling of O and Z.
-        const float m_c = fmaxf(mx0, mx1);
-        const float m_new = (m_c > m_run + kLazyLog2) ? m_c : m_run;
-        const float alpha = ex2(m_run - m_new);
-        if (__any_sync(0xffffffffu, alpha < 1.f)) {
-          for (int c0 = 0; c0 < D; c0 += 16) {
-            float o[16];
-            tmem_ld16(t_o + c0, o);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) o[e] *= alpha;
-            tmem_st16(t_o + c0, o);
-          }
-          float zz[16];
-          tmem_ld16(t_z, zz);
-#pragma unroll
-          for (int e = 0; e < 16; ++e) zz[e] *= alpha;
-          tmem_st16(t_z, zz);
-          tmem_st_wait();
-        }
-        m_run = m_new;
-        auto cpass1 = [&](auto& rg, int c0) __attribute__((always_inline)) {
-          constexpr int W = sizeof(rg) / 4;
-          uint32_t pk[W / 2];
-#pragma unroll
-          for (int u = 0; u < W / 2; ++u)
-            pk[u] = pack_bf16(ex2(u2f(rg[2 * u]) - m_new), ex2(u2f(rg[2 * u + 1]) - m_new));
-          if constexpr (W == 32) tmem_st16u(t_sc + (uint32_t)(c0 >> 1), pk);
-          else tmem_st8(t_sc + (uint32_t)(c0 >> 1), pk);
-        };
-        tmem_walk(t_sc, np16, cpass1, cpass1);
-        tmem_st_wait();
-        tc_fence_before();
-        mbar_arrive(&bars[B_WCREADY]);
-      }
-      if (!ok) break;
-      if (nchunks > 0) {
-        // last chunk of the tile: its value MMA completes the accumulators
-        const int gl = g - 1;
-        if (!AVQ_WAIT(B_CPVDONE + (gl & 1), (gl >> 1) & 1)) break;
-        tc_fence_after();
-      }
-      // ---- Y = O / Z, written row by row (a thread owns one query row: D * 2 contiguous bytes)
-      float zz[16];
-      tmem_ld16(t_z, zz);
-      const float inv = 1.f / zz[0];
-      uint4* yrow = reinterpret_cast<uint4*>(p.Y + ((size_t)bh * p.Nq + i0 + r) * D);
-      auto epi = [&](auto& rg, int c0) __attribute__((always_inline)) {
-        constexpr int W = sizeof(rg) / 4;
-        uint32_t pk[W / 2];
-#pragma unroll
-        for (int e = 0; e < W / 2; ++e) pk[e] = pack_bf16(u2f(rg[2 * e]) * inv, u2f(rg[2 * e + 1]) * inv);
-        if (r < rows_valid) {
-#pragma unroll
-          for (int e = 0; e < W / 8; ++e)
-            yrow[c0 / 8 + e] = make_uint4(pk[4 * e], pk[4 * e + 1], pk[4 * e + 2], pk[4 * e + 3]);
-        }
-      };
-      tmem_walk(t_o, D, epi, epi);
-      tc_fence_before();
-      mbar_arrive(&bars[B_OFREE]);
+      for (int u = 0; u < NQ; ++u) zfull += xz[u * kRows + r];
     }
   }
-#undef AVQ_WAIT
+  // The importances are needed only to choose which parents to refine: with P = 0 (nothing refined) or
+  // P >= M (everything refined) the choice is fixed and the pass is skipped unless the caller wants them.
+  const bool need_w = (P > 0 && P < M) || p.importance_out != nullptr;
+  if (need_w) {
+    const float inv = (r < rows_valid) ? 1.f / zfull : 0.f;
+    // ---- importance: column sums of A_ij / z_i over the 128 rows (32 per warp, then 4 warps)
+    if constexpr ((QW & 31) == 0) {
+#pragma unroll
+      for (int c0 = 0; c0 < QW; c0 += 32) {
+        if (c0 < my_cols) {
+          float v[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = a[c0 + e] * inv;
+          const float colsum = transpose_reduce<32>(v, lane);
+          wpart[q * CT + colbase + c0 + lane] = colsum;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int c0 = 0; c0 < QW; c0 += 16) {
+        if (c0 < my_cols) {
+          float v[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) v[e] = a[c0 + e] * inv;
+          const float colsum = transpose_reduce<16>(v, lane);
+          if ((lane & 1) == 0) wpart[q * CT + colbase + c0 + (lane >> 1)] = colsum;
+        }
+      }
+    }
+  }
+  if (need_w) {
+    __syncthreads();
+    if (tid < M) {
+      const float wj = cnt[tid] * ((wpart[tid] + wpart[CT + tid]) + (wpart[2 * CT + tid] + wpart[3 * CT + tid]));
+      w[tid] = wj;
+      if (p.importance_out) p.importance_out[((size_t)bh * p.nblk + blk) * M + tid] = wj;
+    }
+    __syncthreads();
+  }
 
+  // ---- top-P by rank.  Non-negative floats order like their bit patterns, so the comparisons run on
+  // integers.  gt_j = number of strictly larger importances; parent j is selected if gt_j < P, except
+  // that when a group of EQUAL importances straddles the boundary only its lowest indices are kept.
+  // kT threads share one parent's scan.
+  {
+    const int kT = (kThreads >= 2 * M) ? 2 : 1;          // threads that share one parent's scan
+    const int j = (kT == 2) ? (tid >> 1) : tid, part = (kT == 2) ? (tid & 1) : 0;
+    const uint32_t* keys = reinterpret_cast<const uint32_t*>(w);
+    int* gstar = reinterpret_cast<int*>(&wmask[16]);
+    bool mine = false;
+    if (P >= M) {
+      mine = (j < M) && (part == 0);
+    } else if (P > 0) {
+      int gt = 0;
+      if (j < M) {
+        const uint32_t kj = keys[j];
+        const int span = M / kT, kb = part * span;
+        int g0 = 0, g1 = 0, g2 = 0, g3 = 0;              // four independent counters: no serial add chain
+#pragma unroll 4
+        for (int k = kb; k < kb + span; k += 4) {
+          const uint4 kk = *reinterpret_cast<const uint4*>(keys + k);
+          asm("{\n\t.reg .pred p0, p1, p2, p3;\n\t"
+              "setp.gt.u32 p0, %4, %8;\n\tsetp.gt.u32 p1, %5, %8;\n\t"
+              "setp.gt.u32 p2, %6, %8;\n\tsetp.gt.u32 p3, %7, %8;\n\t"
+              "@p0 add.s32 %0, %0, 1;\n\t@p1 add.s32 %1, %1, 1;\n\t"
+              "@p2 add.s32 %2, %2, 1;\n\t@p3 add.s32 %3, %3, 1;\n\t}"
+              : "+r"(g0), "+r"(g1), "+r"(g2), "+r"(g3)
+              : "r"(kk.x), "r"(kk.y), "r"(kk.z), "r"(kk.w), "r"(kj));
+        }
+        gt = (g0 + g1) + (g2 + g3);
+      }
+      if (kT == 2) gt += __shfl_xor_sync(0xffffffffu, gt, 1);
+      const bool cand = (j < M) && (part == 0) && (gt < P);
+      if (tid == 0) *gstar = 0;
+      const int ncand = __syncthreads_count(cand);
+      mine = cand;
+      if (ncand > P) {                                   // uniform: equal importances straddle the boundary
+        if (cand) atomicMax(gstar, gt);                  // the tied group has the largest gt among candidates
+        __syncthreads();
+        const int g = *gstar;
+        const bool tied = cand && gt == g;
+        const uint32_t beq = __ballot_sync(0xffffffffu, tied);
+        if (lane == 0) wmask[warp] = beq;
+        __syncthreads();
+        int epos = __popc(beq & ((1u << lane) - 1u));
+        for (int u = 0; u < warp; ++u) epos += __popc(wmask[u]);
+        mine = cand && (gt < g || epos < P - g);
+        __syncthreads();
+      }
+    }
+    const uint32_t bal = __ballot_sync(0xffffffffu, mine);
+    if (lane == 0) wmask[warp] = bal;
+    __syncthreads();
+    if (mine) {
+      int pos = __popc(bal & ((1u << lane) - 1u));
+      for (int u = 0; u < warp; ++u) pos += __popc(wmask[u]);
+      sel_list[pos] = j;
+      cntk[j] = 0.f;
+      if (p.topp_out) p.topp_out[((size_t)bh * p.nblk + blk) * P + pos] = j;
+    }
+  }
+  // the output tile of the tile before must have left the child-code buffer before it is refilled (its
+  // store was issued a whole parent pass ago, so this does not wait in practice)
+  if (tid == 0 && store_pending) {
+    tma_store_wait_read();
+    store_pending = false;
+  }
+  __syncthreads();
+
+  // ---- first child chunk: start the asynchronous gather of its codeword rows now; it lands while the
+  // weight conversion below runs
+  const __nv_bfloat16* Cch = p.Cc + (size_t)h * M * C * D;
+  const float* ncb = p.nc + (size_t)bh * M * C;
+  int ncols = min(PC, CHW);
+  int np16 = (ncols + 15) & ~15;
+  // Rows of a chunk, gathered into a K-major / row-per-codeword tile of np16 rows (kSubD sub-tiles of 64
+  // columns): local row e = src[sel_list[(e_first+e)/C] * C + (e_first+e)%C, :]; padding rows are zero.
+  // A thread keeps its 16-byte chunk column and walks down the rows (kThreads is a multiple of the chunks
+  // per row).
+  auto gather_rows = [&](unsigned char* tile, const __nv_bfloat16* src, int e_first) {
+    constexpr int kRowsPerPass = kThreads >> kLogChunks;
+    const int ch = tid & ((1 << kLogChunks) - 1);
+    const uint32_t dst_col = (uint32_t)((ch >> 3) * (np16 * 128));
+    const __nv_bfloat16* src_col = src + ch * 8;
+    for (int row = tid >> kLogChunks; row < np16; row += kRowsPerPass) {
+      unsigned char* dst = tile + dst_col + sw128_offset(row, (ch & 7) * 8);
+      if (row < ncols) {
+        const int e = e_first + row;
+        cp_async16(dst, src_col + (((size_t)sel_list[e >> logC] << logC) + (e & (C - 1))) * D);
+      } else {
+        *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+      }
+    }
+  };
+  auto gather_codes = [&](int e_first) {
+    // the child counts are fetched first so that their latency hides behind the copies
+    float n_child = 0.f;
+    if (tid < ncols) {                                   // CHW <= 128 <= kThreads
+      const int e = e_first + tid;
+      n_child = __ldg(ncb + ((size_t)sel_list[e >> logC] << logC) + (e & (C - 1)));
+    }
+    gather_rows(CC, Cch, e_first);
+    if (tid < CHW) {
+      cntc[tid] = n_child;
+      keepc[tid] = 1.f;
+      biasc[tid] = n_child > 0.f ? 0.f : -INFINITY;
+    }
+  };
+  gather_codes(0);
+
+  // ---- bf16 weights into shared memory (over the dead codebook) + their denominator.  A refined parent
+  // is removed from the numerator by clearing its row of the value tile (d / 8 16-byte stores) and from the
+  // denominator by its zeroed count, so the weights themselves need no mask.
+  mbar_wait(bar_ld1, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);   // value sums have landed
+  for (int u = tid; u < (min(P, M) << kLogChunks); u += kThreads) {
+    const int row = sel_list[u >> kLogChunks], ch = u & ((1 << kLogChunks) - 1);
+    *reinterpret_cast<uint4*>(Vs + (ch >> 3) * (M * 128) + sw128_offset(row, (ch & 7) * 8)) = make_uint4(0, 0, 0, 0);
+  }
+  {
+    float zloc = 0.f;
+#pragma unroll
+    for (int c0 = 0; c0 < QW; c0 += 16) {
+      if (c0 < my_cols) {
+        float am[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) am[e] = a[c0 + e];
+        zloc += store_weights16(CA, r, colbase + c0, cnt + colbase + c0, cntk + colbase + c0, am);
+      }
+    }
+    xz2[cq * kRows + r] = zloc;
+  }
+  cp_async_wait_all();
+  fence_proxy_async();
   tc_fence_before();
   __syncthreads();
-  if (warp == kSelectWarp) tmem_dealloc(tmem_base, p.tmem_cols);
+  float z_run = 0.f;
+#pragma unroll
+  for (int u = 0; u < NQ; ++u) z_run += xz2[u * kRows + r];
+
+  // ---- O = A . Vbar_p, and right behind it the first child chunk's logits
+  if (tid == 0) {
+    tc_fence_after();
+    if (mbar_wait(bar_ld1, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND)) {
+      const uint32_t aa = smem_u32(CA), va = smem_u32(Vs);
+      for (int k = 0; k < M / 16; ++k)
+        umma_bf16(tmem_base + CT, umma_desc_sw128(aa + (k / 4) * kRows * 128 + (k % 4) * 32),
+                  umma_desc_sw128_mn(va + k * 2048, (uint32_t)(M * 128)), idesc_o, k > 0);
+    }
+    umma_commit(bar_pv);
+  }
+  // The child-score MMAs are issued by a lane of another warp: an issuing lane stalls at the tensor pipe's
+  // pace, and two short stalls side by side delay the next CTA-wide barrier less than one long one.
+  if (tid == kScLane && PC > 0) {
+    tc_fence_after();
+    const uint32_t idesc = umma_idesc_bf16(kRows, np16);
+    const uint32_t qa = smem_u32(Qs), ca = smem_u32(CC);
+#pragma unroll
+    for (int k = 0; k < D / 16; ++k)
+      umma_bf16(tmem_base, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
+                umma_desc_sw128(ca + (k / 4) * np16 * 128 + (k % 4) * 32), idesc, k > 0);
+    umma_commit(bar_s);
+  }
+
+  // ---- child chunks
+  const __nv_bfloat16* Vch = p.Vcb + (size_t)bh * M * C * D;
+  for (int e0 = 0; e0 < PC; e0 += CHW) {
+    // The previous second MMA must have released A and Vs before they are rewritten.
+    mbar_wait(bar_pv, ph_pv, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+    ph_pv ^= 1;
+    tc_fence_after();
+    // value rows of this chunk (the same gather as for its codeword rows).  Asynchronous copies: they land
+    // while the chunk's logits are turned into weights.  Padding rows are zero: they meet finite weights.
+    gather_rows(Vs, Vch, e0);
+
+    // ---- child logits: running maximum over non-empty children
+    mbar_wait(bar_s, ph_s, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+    ph_s ^= 1;
+    tc_fence_after();
+    if (tid == 0 && has_next && e0 + CHW >= PC) issue_q(next_tile);   // the last logits are done: Q is dead
+    const int my_c = min(max(np16 - cq * QWC, 0), QWC);
+    float mxc = -INFINITY;
+    for (int c0 = 0; c0 < my_c; c0 += 16) {
+      float s[16];
+      tmem_ld16(t_sc + c0, s);
+      const float4* b4 = reinterpret_cast<const float4*>(biasc + cq * QWC + c0);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float4 b = b4[u];
+        mxc = fmaxf(mxc, fmaxf(s[4 * u] + b.x, s[4 * u + 1] + b.y));
+        mxc = fmaxf(mxc, fmaxf(s[4 * u + 2] + b.z, s[4 * u + 3] + b.w));
+      }
+    }
+    float m_c = mxc * sc;
+    if (NQ > 1) {
+      xm[cq * kRows + r] = m_c;
+      row_sync<NQ>(q);
+#pragma unroll
+      for (int u = 0; u < NQ; ++u) m_c = fmaxf(m_c, xm[u * kRows + r]);
+    }
+    // Any reference value works as long as numerator and denominator share it.  The running one is
+    // kept unless the children exceed it by more than 2^kLazyLog2 (weights up to that factor above 1 are
+    // harmless in fp32 and bf16), which spares most rows the rescaling of O and z.
+    constexpr float kLazyLog2 = 8.f;
+    const float m_new = (m_c > m_run + kLazyLog2) ? m_c : m_run;
+    const float negm = -m_new;
+    // ---- rescale what has been accumulated if this row's maximum moved
+    const float alpha = ex2(m_run + negm);
+    if (__any_sync(0xffffffffu, alpha < 1.f)) {
+      for (int c0 = 0; c0 < D / NQ; c0 += 16) {
+        float o[16];
+        tmem_ld16(t_o + c0, o);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) o[e] *= alpha;
+        tmem_st16(t_o + c0, o);
+      }
+      tmem_st_wait();
+    }
+    z_run *= alpha;
+    m_run = m_new;
+    // ---- bf16 weights of the children over the parents' (consumed) weights
+    {
+      float zloc = 0.f;
+      for (int c0 = 0; c0 < my_c; c0 += 16) {
+        float a[16];
+        tmem_ld16(t_sc + c0, a);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) a[e] = ex2(fminf(fmaf(a[e], sc, negm), kLazyLog2));   // clamp: empty children
+        zloc += store_weights16(CA, r, cq * QWC + c0, cntc + cq * QWC + c0, keepc + cq * QWC + c0, a);
+      }
+      xz2[cq * kRows + r] = zloc;
+    }
+    cp_async_wait_all();
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < NQ; ++u) z_run += xz2[u * kRows + r];
+
+    // ---- O += A_c . Vbar_c; then stage the next chunk's codes (the logits MMA of this chunk is done)
+    const int e_next = e0 + CHW;
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t aa = smem_u32(CA), va = smem_u32(Vs);
+      for (int k = 0; k < np16 / 16; ++k)
+        umma_bf16(tmem_base + CT, umma_desc_sw128(aa + (k / 4) * kRows * 128 + (k % 4) * 32),
+                  umma_desc_sw128_mn(va + k * 2048, (uint32_t)(np16 * 128)), idesc_o, true);
+      umma_commit(bar_pv);
+    }
+    if (e_next < PC) {
+      ncols = min(PC - e_next, CHW);
+      np16 = (ncols + 15) & ~15;
+      gather_codes(e_next);
+      cp_async_wait_all();
+      fence_proxy_async();
+      tc_fence_before();
+      __syncthreads();
+      if (tid == kScLane) {
+        tc_fence_after();
+        const uint32_t idesc = umma_idesc_bf16(kRows, np16);
+        const uint32_t qa = smem_u32(Qs), ca = smem_u32(CC);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)
+          umma_bf16(tmem_base, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
+                    umma_desc_sw128(ca + (k / 4) * np16 * 128 + (k % 4) * 32), idesc, k > 0);
+        umma_commit(bar_s);
+      }
+    }
+  }
+
+  // ---- epilogue: Y = O / z
+  const bool o_ok = mbar_wait(bar_pv, ph_pv, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+  ph_pv ^= 1;
+  tc_fence_after();
+  // the last value MMA has released the weight tile and the value tile: the next tile's codebook and
+  // parent value rows load while this tile's output is written
+  if (tid == 0 && has_next) {
+    issue_cp(next_tile);
+    if (kStageInCC) issue_vp(next_tile);
+  }
+  // The output tile is staged in shared memory in the layout of the Q load and written with TMA tile
+  // stores; rows past Nq are clipped by the tensor map.  Staging area: see the top of the tile loop.
+  unsigned char* stage = kStageInCC ? CC : Vs;
+  if (o_ok) {
+    const float inv = 1.f / z_run;
+    for (int c0 = 0; c0 < D / NQ; c0 += 16) {
+      float o[16];
+      tmem_ld16(t_o + c0, o);
+      uint32_t pk[8];
+#pragma unroll
+      for (int e = 0; e < 16; e += 2) pk[e >> 1] = pack_bf16(o[e] * inv, o[e + 1] * inv);
+      const int col0 = cq * (D / NQ) + c0;
+      unsigned char* sub = stage + (col0 >> 6) * (kRows * 128);
+      *reinterpret_cast<uint4*>(sub + sw128_offset(r, col0 & 63)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      *reinterpret_cast<uint4*>(sub + sw128_offset(r, (col0 & 63) + 8)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+    }
+    fence_proxy_async();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && o_ok) {
+#pragma unroll
+    for (int s2 = 0; s2 < kSubD; ++s2) tma_store_3d(&tmY, stage + s2 * kRows * 128, s2 * 64, i0, bh);
+    tma_store_commit();
+    if (has_next) store_pending = true;                // waited for before the next tile refills CC
+    else tma_store_wait_read();                        // before the CTA may leave
+  }
+  ph_in ^= 1;
+  }   // tiles
+  if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
 }
 
-template <int D, int CT, int CHW, int SB, bool ALIAS>
-avq_status launch_variant(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUtensorMap& tmVpb,
-                          const CUtensorMap& tmCc, const CUtensorMap& tmVcb, AttendParams a, bool chained,
-                          cudaStream_t st) {
-  auto kern = tc_attend_kernel<D, CT, CHW, SB, ALIAS>;
-  constexpr size_t smem = Smem<D, CT, CHW, ALIAS>::kTotal;
-  static_assert(smem <= 227 * 1024, "shared memory");
+size_t attend_smem(int D, int CT, int CHW, int NQ) {
+  const int subA = CT / 64;
+  const size_t ca = (size_t)max(CT * D * 2, subA * kRows * 128);
+  size_t b = (size_t)(D / 64) * kRows * 128 + ca + (size_t)subA * D * 128 + (size_t)CHW * D * 2;
+  b += sizeof(float) * (3 * (size_t)CT + 3 * (size_t)CHW + 256 + 4 * (size_t)CT + 3 * (size_t)NQ * kRows);
+  b += sizeof(int) * 256 + sizeof(uint32_t) * 18 + sizeof(uint64_t) * 5 + 2 * sizeof(uint32_t);
+  return b + 64;
+}
+
+template <int D, int NQ, int CT>
+avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUtensorMap& tmVpb,
+                     const CUtensorMap& tmY, const AttendParams& a, unsigned BH, size_t smem, bool chained,
+                     cudaStream_t st) {
+  auto kern = tc_attend_kernel<D, NQ, CT>;
   // The limit is set once per device and instantiation (setting it again is harmless if two threads race).
-  static bool configured[64] = {};
-  static int sm_count[64] = {};
+  static size_t configured[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return AVQ_ERR_CUDA;
-  const bool cached = dev >= 0 && dev < 64;
-  if (!cached || !configured[dev]) {
+  if (dev < 0 || dev >= 64 || smem > configured[dev]) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return AVQ_ERR_CUDA;
-    if (cached) configured[dev] = true;
+    if (dev >= 0 && dev < 64) configured[dev] = smem;
   }
-  int sms = cached ? sm_count[dev] : 0;
+  // Grid: one wave of CTAs (4 / NQ per SM), each taking every gridDim.x-th tile.
+  static int sm_count[64] = {};
+  int sms = (dev >= 0 && dev < 64) ? sm_count[dev] : 0;
   if (sms <= 0) {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return AVQ_ERR_CUDA;
-    if (cached) sm_count[dev] = sms;
+    if (dev >= 0 && dev < 64) sm_count[dev] = sms;
   }
-  constexpr uint32_t kCols = SB * CT + CHW + D + 16;
-  uint32_t cols = 32;
-  while (cols < kCols) cols <<= 1;
-  a.tmem_cols = cols;
-  // One CTA per SM, each with a contiguous run of tiles (a head's codebook then stays resident).
-  const int ctas = a.total_tiles < sms ? a.total_tiles : sms;
+  int ctas = a.total_tiles;
+  if (ctas > (4 / NQ) * sms) ctas = (4 / NQ) * sms;
+  const dim3 grid((unsigned)ctas);
   // Inside avq_forward (`chained`) the kernel before it in the stream is the aggregate's finalize kernel
   // and Q was complete before the call, so the attention kernel may start as its programmatic dependent.
   // A stand-alone avq_attend is launched plainly: the work before it in the stream may be producing Q.
-  return cuda_ok(launch_pdl(kern, dim3((unsigned)ctas), dim3(kAttendThreads), smem, st, chained, tmQ, tmCp, tmVpb, tmCc,
-                            tmVcb, a));
+  return cuda_ok(launch_pdl(kern, grid, dim3(128 * NQ), smem, st, chained, tmQ, tmCp, tmVpb, tmY, a));
 }
 
 template <int D>
@@ -879,21 +753,13 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
                   const float* nc, const void* Vpb, const void* Vcb, int32_t P, void* Y, int32_t* topp_out,
                   float* importance_out, int32_t* status_word, bool chained, cudaStream_t st) {
   const uint64_t BH = (uint64_t)p.B * p.H;
-  CUtensorMap tmQ, tmCp, tmVpb, tmCc, tmVcb;
-  {
-    // child codewords and child value means as [rows = (head, parent, child), d]: a box is one parent's C rows
-    const uint32_t box[2] = {64, (uint32_t)p.C};
-    const uint64_t dims_c[2] = {(uint64_t)D, (uint64_t)p.H * p.M * p.C};
-    const uint64_t dims_v[2] = {(uint64_t)D, BH * p.M * p.C};
-    avq_status s = make_tmap_bf16(&tmCc, Cc, 2, dims_c, box);
-    if (s != AVQ_OK) return s;
-    s = make_tmap_bf16(&tmVcb, Vcb, 2, dims_v, box);
-    if (s != AVQ_OK) return s;
-  }
+  CUtensorMap tmQ, tmCp, tmVpb, tmY;
   {
     const uint64_t dims[3] = {(uint64_t)D, (uint64_t)p.Nq, BH};
     const uint32_t box[3] = {64, (uint32_t)kRows, 1};
     avq_status s = make_tmap_bf16(&tmQ, Q, 3, dims, box);
+    if (s != AVQ_OK) return s;
+    s = make_tmap_bf16(&tmY, Y, 3, dims, box);
     if (s != AVQ_OK) return s;
   }
   {
@@ -921,33 +787,33 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
   a.nblk = (p.Nq + kRows - 1) / kRows;
   if ((uint64_t)a.nblk * BH > 0x7fffffffull) return AVQ_ERR_UNSUPPORTED;
   a.total_tiles = (int)(a.nblk * BH);
-  a.logC = p.C == 8 ? 3 : 2;
-  a.tmem_cols = 0;
-  a.scale_log2e = p.scale * 1.4426950408889634f;
   const int CT = p.M <= 64 ? 64 : (p.M <= 128 ? 128 : 256);
-  // Variants by TMEM columns (SB*CT + CHW + D + 16 <= 512) and shared memory: two logit buffers up to
-  // CT = 128; at d = 128 the child chunks are 64 columns wide, and with CT = 256 their slots share the
-  // value tile's memory.
-  if constexpr (D == 64) {
-    if (CT == 64) return launch_variant<D, 64, 128, 2, false>(tmQ, tmCp, tmVpb, tmCc, tmVcb, a, chained, st);
-    if (CT == 128) return launch_variant<D, 128, 128, 2, false>(tmQ, tmCp, tmVpb, tmCc, tmVcb, a, chained, st);
-    return launch_variant<D, 256, 128, 1, false>(tmQ, tmCp, tmVpb, tmCc, tmVcb, a, chained, st);
-  } else {
-    if (CT == 64) return launch_variant<D, 64, 64, 2, false>(tmQ, tmCp, tmVpb, tmCc, tmVcb, a, chained, st);
-    if (CT == 128) return launch_variant<D, 128, 64, 2, false>(tmQ, tmCp, tmVpb, tmCc, tmVcb, a, chained, st);
-    return launch_variant<D, 256, 64, 1, true>(tmQ, tmCp, tmVpb, tmCc, tmVcb, a, chained, st);
+  const int CHW = CT < 128 ? CT : 128;
+  a.logC = p.C == 8 ? 3 : 2;
+  uint32_t cols = 32;
+  while ((int)cols < CT + D) cols <<= 1;
+  a.tmem_cols = cols;
+  a.scale_log2e = p.scale * 1.4426950408889634f;
+  const int NQ = (D == 64) ? (CT == 64 ? 1 : (CT == 128 ? 2 : 4)) : (CT == 64 ? 2 : 4);
+  const size_t smem = attend_smem(D, CT, CHW, NQ);
+  // Threads per query row follow from how many CTAs can share an SM (TMEM columns, shared memory):
+  // four small CTAs of 128 threads, two of 256, or one of 512.
+  const unsigned bh = (unsigned)BH;
+  if (D == 64) {
+    if (CT == 64) return launch_nq<D, 1, 64>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
+    if (CT == 128) return launch_nq<D, 2, 128>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
+    return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
   }
+  if (CT == 64) return launch_nq<D, 2, 64>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
+  if (CT == 128) return launch_nq<D, 4, 128>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
+  return launch_nq<D, 4, 256>(tmQ, tmCp, tmVpb, tmY, a, bh, smem, chained, st);
 }
 
 }  // namespace
 
-// Parent tiles of up to 128 codewords leave room for several small CTAs per SM (avq_tc_attend_small.cu);
-// larger ones take the whole SM and run the warp-specialised kernel above.
 avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc, const float* np_,
                      const float* nc, const void* Vpb, const void* Vcb, int32_t P, void* Y, int32_t* topp_out,
                      float* importance_out, int32_t* status_word, bool chained, cudaStream_t st) {
-  if (p.M <= 128)
-    return tc_attend_small(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, P, Y, topp_out, importance_out, status_word, chained, st);
   return p.d == 64 ? launch<64>(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, P, Y, topp_out, importance_out, status_word, chained, st)
                    : launch<128>(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, P, Y, topp_out, importance_out, status_word, chained, st);
 }
