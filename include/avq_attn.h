@@ -150,6 +150,21 @@ AVQ_API avq_status avq_forward(const avq_problem* prob, const void* Q, const voi
                        int32_t* topp_out, float* importance_out, void* workspace,
                        size_t workspace_bytes, void* stream);
 
+/* avq_forward over query tiles that follow a caller-supplied token order (Sec. "Vector Quantization for
+ * (A)VQ-Attention": tokens of an image are reordered along a space-filling curve so that a query tile holds
+ * neighbouring tokens; building the curve is the caller's business).  perm: int32 [Nq], a permutation of
+ * 0..Nq-1 shared by every (batch, head): tile t holds the queries perm[t*block_q .. (t+1)*block_q).  Only
+ * the grouping of the queries changes the result (sums and counts over keys do not depend on their order),
+ * so K and V are used as given.  Y, topp_out and importance_out as in avq_forward, with Y rows in the
+ * caller's ORIGINAL order and tile t of the optional outputs referring to the permuted tile t.
+ * Needs avq_workspace_bytes_permuted() bytes (the forward's workspace plus two [B,H,Nq,d] buffers).  An
+ * entry of perm outside [0, Nq) is skipped and reported by avq_check() as AVQ_ERR_INDEX. */
+AVQ_API size_t avq_workspace_bytes_permuted(const avq_problem* prob, int32_t P, int32_t block_q);
+AVQ_API avq_status avq_forward_permuted(const avq_problem* prob, const void* Q, const void* K, const void* V,
+                                const void* Cp, const void* Cc, int32_t P, int32_t block_q,
+                                const int32_t* perm, void* Y, int32_t* topp_out, float* importance_out,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
 /* Stage 3 alone: the attention pass of avq_forward over a workspace that a previous
  * avq_forward call with the same `prob`, P and block_q (and the same K, V, Cp, Cc) filled.
  * Reads the aggregates from the workspace, recomputes Y (and the optional outputs) for Q.

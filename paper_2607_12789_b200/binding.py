@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "AVQ_OK", 1: "AVQ_ERR_NULL", 2: "AVQ_ERR_SHAPE", 3: "AVQ_ERR_
 
 EXPORTS = ("avq_workspace_bytes", "avq_assign", "avq_aggregate", "avq_forward", "avq_forward_host", "avq_attend",
            "avq_workspace_layout", "avq_check", "avq_status_string", "avq_version", "avq_forward_static",
-           "avq_check_static", "avq_static_workspace_bytes")
+           "avq_check_static", "avq_static_workspace_bytes", "avq_workspace_bytes_permuted",
+           "avq_forward_permuted")
 
 
 class AvqProblem(ctypes.Structure):
@@ -68,6 +69,9 @@ def lib() -> ctypes.CDLL:
         L.avq_forward_static.argtypes = [pp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
         L.avq_check_static.restype, L.avq_check_static.argtypes = i32, [vp]
         L.avq_static_workspace_bytes.restype, L.avq_static_workspace_bytes.argtypes = sz, []
+        L.avq_workspace_bytes_permuted.restype, L.avq_workspace_bytes_permuted.argtypes = sz, [pp, i32, i32]
+        L.avq_forward_permuted.restype = i32
+        L.avq_forward_permuted.argtypes = [pp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
         L.avq_status_string.restype, L.avq_status_string.argtypes = ctypes.c_char_p, [i32]
         L.avq_version.restype, L.avq_version.argtypes = i32, []
         _lib = L
@@ -232,6 +236,28 @@ def forward(Q, K, V, Cp, Cc, P: int, block_q: int, scale=None, flags: int = 0, a
     if aux:
         return Y, f.topp, f.importance, f.intermediates()
     return Y
+
+
+def forward_permuted(Q, K, V, Cp, Cc, P: int, block_q: int, perm, scale=None, flags: int = 0):
+    """avq_forward_permuted: query tiles follow ``perm`` (int32 [Nq]).  Returns (Y, topp, importance, status)
+    where status is what avq_check reports after the call (0, or 8 if perm held an index out of range)."""
+    _chk(Q, K, V, Cp, Cc, perm)
+    prob = _problem_from(Q, K, Cp, Cc, scale, flags)
+    B, H, Nq, d = Q.shape
+    nblk = (Nq + block_q - 1) // block_q
+    nbytes = int(lib().avq_workspace_bytes_permuted(ctypes.byref(prob), P, block_q))
+    if nbytes == 0:
+        raise AvqError(lib().avq_workspace_layout(ctypes.byref(prob), P, block_q, None, None, None, None, None, None)
+                       or 3, "avq_workspace_bytes_permuted")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=Q.device)
+    Y = torch.zeros_like(Q)
+    topp = torch.empty((B, H, nblk, P), dtype=torch.int32, device=Q.device)
+    imp = torch.empty((B, H, nblk, prob.M), dtype=torch.float32, device=Q.device)
+    st = lib().avq_forward_permuted(ctypes.byref(prob), _ptr(Q), _ptr(K), _ptr(V), _ptr(Cp), _ptr(Cc), P, block_q,
+                                    _ptr(perm), _ptr(Y), _ptr(topp), _ptr(imp), _ptr(ws), nbytes, _stream())
+    if st != 0:
+        raise AvqError(st, "avq_forward_permuted")
+    return Y, topp, imp, int(lib().avq_check(_ptr(ws), _stream()))
 
 
 def forward_static(Q, K, V, Cp, Cc, P: int, block_q: int, scale=None, flags: int = 0, aux: bool = False):
