@@ -25,6 +25,11 @@ What each function follows in the paper:
                          (Sec. 3.2 regrouping + the post-refinement sum of the appendix
                          "Correcting Attention Derivation": ``A_p Vbar_stay + sum_c A_c Vbar_c``).
 
+* ``codebook_update``  - appendix "Codeword Clustering During Training": EMA statistics of the
+                         keys assigned to every parent and child, parents moved to their EMA mean,
+                         children to the mass-weighted projection of their EMA means onto the
+                         parent = mean(children) constraint (Eq. "child_constraint_solve").
+
 Two child-assignment rules are implemented.  REPLACE (default): every key goes
 to the nearest child of its parent.  PARENT_STAYS (Algorithm 1's masked scatter):
 a key moves to that child only if it is strictly closer than the parent.
@@ -33,6 +38,10 @@ Readings taken where the paper is silent: ties go to the lowest index
 everywhere; the logit scale is an explicit argument; the importance denominator
 is the exact parent-pass one; query blocks are contiguous ranges of ``block_q``
 queries inside one (batch, head), the last one may be short.
+
+``codebook_update`` reading where the paper is silent: a code whose EMA mass is (still) zero keeps
+its previous position as its "unconstrained mean" and enters the projection with a mass floor of
+``mass_floor`` (it has no data to resist the displacement, so it absorbs the residual).
 
 Pins (tests/test_oracle_*.py): brute-force loops on tiny inputs, closed forms,
 conservation laws, the exact-attention special case checked against
@@ -294,3 +303,52 @@ def forward(Q, K, V, Cp, Cc, P: int, block_q: int, scale: float, parent_stays: b
     for k in ("parent_idx", "child_idx", "parent_margin", "child_margin", "stay_margin"):
         out[k] = np.stack([np.stack([res[b][h]["assignment"][k] for h in range(H)]) for b in range(B)])
     return out
+
+
+# --------------------------------------------------------------------------- codebook update (training)
+def codebook_update(K, Cp, Cc, Sp, Np, Sc, Nc, decay: float, parent_stays: bool = False,
+                    mass_floor: float = 1e-6):
+    """One codebook update from a batch of keys (appendix "Codeword Clustering During Training").
+
+    K [B,H,N,d]; Cp [H,M,d], Cc [H,M,C,d] the current codebooks (one per head, shared over the batch);
+    Sp [H,M,d], Np [H,M], Sc [H,M,C,d], Nc [H,M,C] the EMA statistics before the update.
+
+    1. keys are assigned with the current codebooks (``assign_head``); a parent collects every key assigned
+       to it, a child the keys that moved to it;
+    2. ``S <- decay * S + (1 - decay) * sum of the code's keys``, ``N <- decay * N + (1 - decay) * count``;
+    3. parents: ``Cp' = Sp / Np``; children: unconstrained means ``Mc = Sc / Nc``, then
+       ``Cc' = Mc - delta / (Nc * sigma)`` with ``delta = sum_c Mc - C * Cp'`` and ``sigma = sum_c 1 / Nc``
+       (Eq. "child_constraint_solve"), which restores ``mean_c Cc' = Cp'``.
+
+    Returns a dict with the new Sp, Np, Sc, Nc, Cp, Cc (float64).
+    """
+    K = np.asarray(K, dtype=F64)
+    Cp = np.asarray(Cp, dtype=F64)
+    Cc = np.asarray(Cc, dtype=F64)
+    B, H, N, d = K.shape
+    M, C = Cc.shape[1], Cc.shape[2]
+    sum_p = np.zeros((H, M, d))
+    cnt_p = np.zeros((H, M))
+    sum_c = np.zeros((H, M, C, d))
+    cnt_c = np.zeros((H, M, C))
+    for b in range(B):
+        for h in range(H):
+            a = assign_head(K[b, h], Cp[h], Cc[h], parent_stays)
+            kp, n_p, kc, n_c = aggregate_head(K[b, h], a["parent_idx"], a["child_idx"], M, C)
+            sum_p[h] += kp
+            cnt_p[h] += n_p
+            sum_c[h] += kc
+            cnt_c[h] += n_c
+    Sp2 = decay * np.asarray(Sp, dtype=F64) + (1.0 - decay) * sum_p
+    Np2 = decay * np.asarray(Np, dtype=F64) + (1.0 - decay) * cnt_p
+    Sc2 = decay * np.asarray(Sc, dtype=F64) + (1.0 - decay) * sum_c
+    Nc2 = decay * np.asarray(Nc, dtype=F64) + (1.0 - decay) * cnt_c
+    has_p = Np2 > mass_floor
+    Cp2 = np.where(has_p[..., None], Sp2 / np.where(has_p, Np2, 1.0)[..., None], Cp)
+    has_c = Nc2 > mass_floor
+    Mc = np.where(has_c[..., None], Sc2 / np.where(has_c, Nc2, 1.0)[..., None], Cc)
+    mass = np.maximum(Nc2, mass_floor)
+    delta = Mc.sum(axis=2) - C * Cp2                                  # [H,M,d]
+    sigma = (1.0 / mass).sum(axis=2)                                  # [H,M]
+    Cc2 = Mc - delta[:, :, None, :] / (mass * sigma[:, :, None])[..., None]
+    return dict(Sp=Sp2, Np=Np2, Sc=Sc2, Nc=Nc2, Cp=Cp2, Cc=Cc2)
