@@ -165,6 +165,25 @@ AVQ_API avq_status avq_forward_permuted(const avq_problem* prob, const void* Q, 
                                 const int32_t* perm, void* Y, int32_t* topp_out, float* importance_out,
                                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* One training-time update of the codebooks from a batch of keys (appendix "Codeword Clustering During
+ * Training").  The keys are assigned under the current codebooks (as in avq_assign, honouring
+ * AVQ_FLAG_PARENT_STAYS); every parent and child adds the sum and the number of its keys, over the whole batch,
+ * to its exponential-moving-average statistics,  S <- decay*S + (1-decay)*sum,  N <- decay*N + (1-decay)*count;
+ * a parent moves to Sp/Np; the children of a parent move to
+ *     Cc' = Mc - delta / (Nc * sigma),   Mc = Sc/Nc,  delta = sum_c Mc - C*Cp',  sigma = sum_c 1/Nc
+ * (Eq. "child_constraint_solve"), the mass-weighted least-squares projection onto  mean_c Cc' = Cp'.
+ * A code whose EMA mass is below 1e-6 keeps its previous position as its mean and enters the projection
+ * with that floor as its mass (the appendix does not say; with no data it absorbs the residual).
+ *   K [B,H,Nk,d];  Cp [H,M,d], Cc [H,M,C,d] current codebooks (read only)
+ *   Sp [H,M,d], Np [H,M], Sc [H,M,C,d], Nc [H,M,C]   float32 EMA statistics, updated in place
+ *   Cp_out, Cc_out   the new codebooks, dtype of K (bfloat16 rounding perturbs the constraint by an ulp)
+ *   workspace        avq_codebook_update_workspace_bytes() bytes, 256-byte aligned
+ * C <= 16.  Uses B, H, Nk, d, M, C, dtype, flags of `prob`. */
+AVQ_API size_t avq_codebook_update_workspace_bytes(const avq_problem* prob);
+AVQ_API avq_status avq_codebook_update(const avq_problem* prob, const void* K, const void* Cp, const void* Cc,
+                               float decay, float* Sp, float* Np, float* Sc, float* Nc, void* Cp_out,
+                               void* Cc_out, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Stage 3 alone: the attention pass of avq_forward over a workspace that a previous
  * avq_forward call with the same `prob`, P and block_q (and the same K, V, Cp, Cc) filled.
  * Reads the aggregates from the workspace, recomputes Y (and the optional outputs) for Q.

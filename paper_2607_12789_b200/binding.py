@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "AVQ_OK", 1: "AVQ_ERR_NULL", 2: "AVQ_ERR_SHAPE", 3: "AVQ_ERR_
 EXPORTS = ("avq_workspace_bytes", "avq_assign", "avq_aggregate", "avq_forward", "avq_forward_host", "avq_attend",
            "avq_workspace_layout", "avq_check", "avq_status_string", "avq_version", "avq_forward_static",
            "avq_check_static", "avq_static_workspace_bytes", "avq_workspace_bytes_permuted",
-           "avq_forward_permuted")
+           "avq_forward_permuted", "avq_codebook_update_workspace_bytes", "avq_codebook_update")
 
 
 class AvqProblem(ctypes.Structure):
@@ -72,6 +72,9 @@ def lib() -> ctypes.CDLL:
         L.avq_workspace_bytes_permuted.restype, L.avq_workspace_bytes_permuted.argtypes = sz, [pp, i32, i32]
         L.avq_forward_permuted.restype = i32
         L.avq_forward_permuted.argtypes = [pp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.avq_codebook_update_workspace_bytes.restype, L.avq_codebook_update_workspace_bytes.argtypes = sz, [pp]
+        L.avq_codebook_update.restype = i32
+        L.avq_codebook_update.argtypes = [pp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.avq_status_string.restype, L.avq_status_string.argtypes = ctypes.c_char_p, [i32]
         L.avq_version.restype, L.avq_version.argtypes = i32, []
         _lib = L
@@ -258,6 +261,20 @@ def forward_permuted(Q, K, V, Cp, Cc, P: int, block_q: int, perm, scale=None, fl
     if st != 0:
         raise AvqError(st, "avq_forward_permuted")
     return Y, topp, imp, int(lib().avq_check(_ptr(ws), _stream()))
+
+
+def codebook_update(K, Cp, Cc, Sp, Np, Sc, Nc, decay: float, flags: int = 0):
+    """avq_codebook_update: EMA statistics (updated in place) and the new codebooks (Cp', Cc')."""
+    _chk(K, Cp, Cc, Sp, Np, Sc, Nc)
+    prob = _problem_from(None, K, Cp, Cc, 1.0, flags)
+    nbytes = int(lib().avq_codebook_update_workspace_bytes(ctypes.byref(prob)))
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=K.device)
+    Cp2, Cc2 = torch.empty_like(Cp), torch.empty_like(Cc)
+    st = lib().avq_codebook_update(ctypes.byref(prob), _ptr(K), _ptr(Cp), _ptr(Cc), decay, _ptr(Sp), _ptr(Np),
+                                   _ptr(Sc), _ptr(Nc), _ptr(Cp2), _ptr(Cc2), _ptr(ws), ws.numel(), _stream())
+    if st != 0:
+        raise AvqError(st, "avq_codebook_update")
+    return Cp2, Cc2
 
 
 def forward_static(Q, K, V, Cp, Cc, P: int, block_q: int, scale=None, flags: int = 0, aux: bool = False):
