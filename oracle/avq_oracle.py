@@ -25,6 +25,12 @@ What each function follows in the paper:
                          (Sec. 3.2 regrouping + the post-refinement sum of the appendix
                          "Correcting Attention Derivation": ``A_p Vbar_stay + sum_c A_c Vbar_c``).
 
+* ``importance_block_tiled`` - appendix "Computing Importance with Tiled Codewords": the parents are
+                         visited in tiles; a tile's importances use the denominator seen so far,
+                         extrapolated by key counts (Eq. "aproxdenom", Eq. "codewordimportance").
+* ``capture``          - the fraction of a block's TRUE attention mass (exact softmax over the
+                         original keys) that falls on keys of the selected parents (the measure of
+                         Table "tiled_capture").
 * ``codebook_update``  - appendix "Codeword Clustering During Training": EMA statistics of the
                          keys assigned to every parent and child, parents moved to their EMA mean,
                          children to the mass-weighted projection of their EMA means onto the
@@ -170,6 +176,66 @@ def importance_block(Qb, Cp, n_p, scale: float):
     return w, s, m, z
 
 
+def importance_block_tiled(Qb, Cp, n_p, scale: float, tile_m: int, n_keys: float | None = None):
+    """Importance when the parents are visited in tiles of ``tile_m`` codewords, in index order
+    (appendix "Computing Importance with Tiled Codewords").
+
+    After tiles ``t <= J`` the denominator of row i is known only over the visited codewords,
+    ``Zpart_i(J) = sum_{t<=J} sum_{j in t} A_ij n_j``; it is extrapolated by key counts,
+    ``Ztilde_i(J) = N / N_seen(J) * Zpart_i(J)`` (Eq. "aproxdenom"), and the codewords of tile J get
+    ``w_j = sum_i A_ij n_j / Ztilde_i(J)`` (Eq. "codewordimportance").  The ratio does not depend on the
+    stabiliser, so the plain row maximum over non-empty parents is used.  A tile reached before any key has
+    been seen holds only empty parents: their importance is 0.  ``n_keys`` defaults to ``sum(n_p)``.
+    """
+    Qb = np.asarray(Qb, dtype=F64)
+    Cp = np.asarray(Cp, dtype=F64)
+    n_p = np.asarray(n_p, dtype=F64)
+    M = n_p.shape[0]
+    N = float(n_p.sum()) if n_keys is None else float(n_keys)
+    s = scale * (Qb @ Cp.T)
+    live = n_p > 0
+    m = np.max(np.where(live[None, :], s, -np.inf), axis=1)
+    An = np.where(live[None, :], np.exp(s - m[:, None]), 0.0) * n_p[None, :]     # A_ij n_j
+    w = np.zeros(M)
+    zpart = np.zeros(Qb.shape[0])
+    n_seen = 0.0
+    for j0 in range(0, M, tile_m):
+        j1 = min(M, j0 + tile_m)
+        zpart = zpart + An[:, j0:j1].sum(axis=1)
+        n_seen += float(n_p[j0:j1].sum())
+        if n_seen > 0:
+            ztilde = (N / n_seen) * zpart
+            w[j0:j1] = (An[:, j0:j1] / ztilde[:, None]).sum(axis=0)
+    return w
+
+
+def capture(Qb, K, parent_idx, selected, scale: float) -> float:
+    """Share of the block's true attention mass on the keys whose parent is in ``selected``: exact softmax of
+    the block's queries over the ORIGINAL keys, summed over those keys and averaged over the queries."""
+    Qb = np.asarray(Qb, dtype=F64)
+    K = np.asarray(K, dtype=F64)
+    s = scale * (Qb @ K.T)
+    s -= s.max(axis=1, keepdims=True)
+    E = np.exp(s)
+    E /= E.sum(axis=1, keepdims=True)
+    hit = np.isin(parent_idx, np.asarray(selected, dtype=np.int64))
+    return float(E[:, hit].sum(axis=1).mean())
+
+
+def exact_selection(Qb, K, parent_idx, M: int, P: int, scale: float):
+    """The P parents whose keys receive the most true attention mass from the block (the "exact" column of
+    Table "tiled_capture"), ascending."""
+    Qb = np.asarray(Qb, dtype=F64)
+    K = np.asarray(K, dtype=F64)
+    s = scale * (Qb @ K.T)
+    s -= s.max(axis=1, keepdims=True)
+    E = np.exp(s)
+    E /= E.sum(axis=1, keepdims=True)
+    mass = np.zeros(M)
+    np.add.at(mass, parent_idx, E.sum(axis=0))
+    return top_p(mass, P)[0]
+
+
 def top_p(w, P: int):
     """Indices of the P largest importances, lowest index first among equals.
 
@@ -244,13 +310,14 @@ def forward_block_factorised(Qb, Cp, Cc, Vp, n_p, Vc, n_c, selected, scale: floa
 
 # --------------------------------------------------------------------------- forward, one head / all heads
 def forward_head(Q, K, V, Cp, Cc, P: int, block_q: int, scale: float, parent_stays: bool = False,
-                 form: str = "dense", blocks=None, assignment=None):
+                 form: str = "dense", blocks=None, assignment=None, tile_m: int | None = None):
     """AVQ-attention forward for one (batch, head).
 
     Q [Nq,d], K,V [Nk,d], Cp [M,d], Cc [M,C,d].  ``form`` is "dense" (definition) or
     "factorised".  ``blocks`` optionally restricts the evaluation to some query-block
     indices (rows of other blocks are left NaN).  ``assignment`` may carry a
-    previously computed ``assign_head`` result for these keys.
+    previously computed ``assign_head`` result for these keys.  ``tile_m`` switches the selection to the
+    tiled importance (the output is still exact for the parents that selection refines).
 
     Returns a dict: Y [Nq,d]; selected [nblk,P] (ascending, -1 rows for skipped
     blocks); importance [nblk,M]; topp_margin [nblk]; plus the assignment dict and
@@ -274,7 +341,10 @@ def forward_head(Q, K, V, Cp, Cc, P: int, block_q: int, scale: float, parent_sta
     for t in todo:
         i0, i1 = t * block_q, min(Nq, (t + 1) * block_q)
         Qb = Q[i0:i1]
-        w, _, _, _ = importance_block(Qb, Cp64, n_p, scale)
+        if tile_m is None:
+            w, _, _, _ = importance_block(Qb, Cp64, n_p, scale)
+        else:
+            w = importance_block_tiled(Qb, Cp64, n_p, scale, tile_m, n_keys=float(np.asarray(K).shape[0]))
         sel, mg = top_p(w, P)
         importance[t] = w
         selected[t] = sel
@@ -290,10 +360,11 @@ def forward_head(Q, K, V, Cp, Cc, P: int, block_q: int, scale: float, parent_sta
 
 
 def forward(Q, K, V, Cp, Cc, P: int, block_q: int, scale: float, parent_stays: bool = False,
-            form: str = "dense"):
+            form: str = "dense", tile_m: int | None = None):
     """All (batch, head) pairs.  Q,K,V [B,H,N,d]; Cp [H,M,d]; Cc [H,M,C,d] (one codebook per head)."""
     B, H = Q.shape[:2]
-    res = [[forward_head(Q[b, h], K[b, h], V[b, h], Cp[h], Cc[h], P, block_q, scale, parent_stays, form)
+    res = [[forward_head(Q[b, h], K[b, h], V[b, h], Cp[h], Cc[h], P, block_q, scale, parent_stays, form,
+                         tile_m=tile_m)
             for h in range(H)] for b in range(B)]
 
     def stack(key):
