@@ -165,6 +165,20 @@ AVQ_API avq_status avq_forward_permuted(const avq_problem* prob, const void* Q, 
                                 const int32_t* perm, void* Y, int32_t* topp_out, float* importance_out,
                                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* avq_forward with the parents visited in tiles of tile_m codewords, for codebooks too large to score in one
+ * tile (appendix "Computing Importance with Tiled Codewords").  The codewords of tile J get their importance
+ * from the part of the softmax denominator seen up to that tile, extrapolated by key counts:
+ *     Ztilde_i(J) = Nk / N_seen(J) * sum_{t<=J} sum_{j in t} A_ij n_j          (Eq. "aproxdenom")
+ *     w_j = sum_i A_ij n_j / Ztilde_i(J),  j in J                              (Eq. "codewordimportance")
+ * and the P parents with the largest w are refined.  The output is the exact refined attention for that
+ * selection; only the selection (and importance_out) differs from avq_forward.  tile_m: a multiple of 32;
+ * tile_m >= M reproduces avq_forward.  Runs the CUDA-core kernels for either dtype (M up to 1024); the
+ * workspace is that of avq_forward for the same problem with AVQ_FLAG_SIMT set. */
+AVQ_API avq_status avq_forward_tiled(const avq_problem* prob, const void* Q, const void* K, const void* V,
+                             const void* Cp, const void* Cc, int32_t P, int32_t block_q, int32_t tile_m,
+                             void* Y, int32_t* topp_out, float* importance_out, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
 /* One training-time update of the codebooks from a batch of keys (appendix "Codeword Clustering During
  * Training").  The keys are assigned under the current codebooks (as in avq_assign, honouring
  * AVQ_FLAG_PARENT_STAYS); every parent and child adds the sum and the number of its keys, over the whole batch,

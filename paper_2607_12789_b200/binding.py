@@ -23,7 +23,8 @@ STATUS_NAMES = {0: "AVQ_OK", 1: "AVQ_ERR_NULL", 2: "AVQ_ERR_SHAPE", 3: "AVQ_ERR_
 EXPORTS = ("avq_workspace_bytes", "avq_assign", "avq_aggregate", "avq_forward", "avq_forward_host", "avq_attend",
            "avq_workspace_layout", "avq_check", "avq_status_string", "avq_version", "avq_forward_static",
            "avq_check_static", "avq_static_workspace_bytes", "avq_workspace_bytes_permuted",
-           "avq_forward_permuted", "avq_codebook_update_workspace_bytes", "avq_codebook_update")
+           "avq_forward_permuted", "avq_codebook_update_workspace_bytes", "avq_codebook_update",
+           "avq_forward_tiled")
 
 
 class AvqProblem(ctypes.Structure):
@@ -72,6 +73,8 @@ def lib() -> ctypes.CDLL:
         L.avq_workspace_bytes_permuted.restype, L.avq_workspace_bytes_permuted.argtypes = sz, [pp, i32, i32]
         L.avq_forward_permuted.restype = i32
         L.avq_forward_permuted.argtypes = [pp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.avq_forward_tiled.restype = i32
+        L.avq_forward_tiled.argtypes = [pp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
         L.avq_codebook_update_workspace_bytes.restype, L.avq_codebook_update_workspace_bytes.argtypes = sz, [pp]
         L.avq_codebook_update.restype = i32
         L.avq_codebook_update.argtypes = [pp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -261,6 +264,27 @@ def forward_permuted(Q, K, V, Cp, Cc, P: int, block_q: int, perm, scale=None, fl
     if st != 0:
         raise AvqError(st, "avq_forward_permuted")
     return Y, topp, imp, int(lib().avq_check(_ptr(ws), _stream()))
+
+
+def forward_tiled(Q, K, V, Cp, Cc, P: int, block_q: int, tile_m: int, scale=None, flags: int = 0):
+    """avq_forward_tiled: selection from the tiled importance.  Returns (Y, topp, importance)."""
+    _chk(Q, K, V, Cp, Cc)
+    prob = _problem_from(Q, K, Cp, Cc, scale, flags | FLAG_SIMT)
+    B, H, Nq, d = Q.shape
+    nblk = (Nq + block_q - 1) // block_q
+    nbytes = workspace_bytes(prob, P, block_q)
+    if nbytes == 0:
+        raise AvqError(lib().avq_workspace_layout(ctypes.byref(prob), P, block_q, None, None, None, None, None, None)
+                       or 3, "avq_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=Q.device)
+    Y = torch.empty_like(Q)
+    topp = torch.empty((B, H, nblk, P), dtype=torch.int32, device=Q.device)
+    imp = torch.empty((B, H, nblk, prob.M), dtype=torch.float32, device=Q.device)
+    st = lib().avq_forward_tiled(ctypes.byref(prob), _ptr(Q), _ptr(K), _ptr(V), _ptr(Cp), _ptr(Cc), P, block_q,
+                                 tile_m, _ptr(Y), _ptr(topp), _ptr(imp), _ptr(ws), nbytes, _stream())
+    if st != 0:
+        raise AvqError(st, "avq_forward_tiled")
+    return Y, topp, imp
 
 
 def codebook_update(K, Cp, Cc, Sp, Np, Sc, Nc, decay: float, flags: int = 0):

@@ -48,7 +48,7 @@ avq_status validate_forward(const avq_problem* p, int32_t P, int32_t block_q) {
   } else {
     if (block_q > 256) return AVQ_ERR_UNSUPPORTED;
     if ((int64_t)p->M + (int64_t)P * p->C > 8192) return AVQ_ERR_UNSUPPORTED;
-    if (simt_attend_smem_bytes(p->d, p->M, p->C, P, block_q) > kSimtAttendSmemLimit) return AVQ_ERR_UNSUPPORTED;
+    if (simt_attend_smem_bytes(p->d, p->M, p->C, P, block_q, 0) > kSimtAttendSmemLimit) return AVQ_ERR_UNSUPPORTED;
   }
   return AVQ_OK;
 }
@@ -153,7 +153,7 @@ avq_status attend_stage(const avq_problem& p, const Regions& r, const void* Q, c
   if (use_tensor_path(p))
     return tc_attend(p, Q, Cp, Cc, r.np_, r.nc, r.Vpb, r.Vcb, P, Y, topp_out, importance_out, r.status_word,
                      chained, st);
-  return simt_attend(p, Q, Cp, Cc, r.Vp, r.np_, r.Vc, r.nc, P, block_q, Y, topp_out, importance_out, st);
+  return simt_attend(p, Q, Cp, Cc, r.Vp, r.np_, r.Vc, r.nc, P, block_q, Y, topp_out, importance_out, 0, st);
 }
 avq_status check_workspace(const avq_problem* prob, int32_t P, int32_t block_q, void* workspace,
                            size_t workspace_bytes, Layout* L) {
@@ -194,6 +194,34 @@ avq_status avq_forward(const avq_problem* prob, const void* Q, const void* K, co
   }
   if (s != AVQ_OK) return s;
   return attend_stage(p, r, Q, Cp, Cc, P, block_q, Y, topp_out, importance_out, true, st);
+}
+
+avq_status avq_forward_tiled(const avq_problem* prob, const void* Q, const void* K, const void* V,
+                             const void* Cp, const void* Cc, int32_t P, int32_t block_q, int32_t tile_m,
+                             void* Y, int32_t* topp_out, float* importance_out, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+  if (!prob) return AVQ_ERR_NULL;
+  avq_problem p = *prob;
+  p.flags |= AVQ_FLAG_SIMT;                        // the tiled importance lives in the CUDA-core attention kernel
+  avq_status s = validate_forward(&p, P, block_q);
+  if (s != AVQ_OK) return s;
+  if (tile_m < 32 || tile_m % 32 != 0) return AVQ_ERR_SHAPE;
+  if (simt_attend_smem_bytes(p.d, p.M, p.C, P, block_q, tile_m) > kSimtAttendSmemLimit) return AVQ_ERR_UNSUPPORTED;
+  if (!Q || !K || !V || !Cp || !Cc || !Y) return AVQ_ERR_NULL;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(Cp) || !aligned16(Cc) || !aligned16(Y) ||
+      !aligned16(topp_out) || !aligned16(importance_out))
+    return AVQ_ERR_ALIGN;
+  Layout L;
+  s = check_workspace(&p, P, block_q, workspace, workspace_bytes, &L);
+  if (s != AVQ_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Regions r = carve(workspace, L);
+  if (cudaMemsetAsync(r.status_word, 0, 256, st) != cudaSuccess) return AVQ_ERR_CUDA;
+  s = simt_assign(p, K, Cp, Cc, r.pidx, r.cidx, st);
+  if (s != AVQ_OK) return s;
+  s = simt_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, st);
+  if (s != AVQ_OK) return s;
+  return simt_attend(p, Q, Cp, Cc, r.Vp, r.np_, r.Vc, r.nc, P, block_q, Y, topp_out, importance_out, tile_m, st);
 }
 
 avq_status avq_attend(const avq_problem* prob, const void* Q, const void* Cp, const void* Cc, int32_t P,

@@ -47,10 +47,10 @@ avq_status simt_aggregate(const avq_problem& p, const void* V, const int32_t* pa
 avq_status simt_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc,
                        const float* Vp, const float* np_, const float* Vc, const float* nc, int32_t P,
                        int32_t block_q, void* Y, int32_t* topp_out, float* importance_out,
-                       cudaStream_t st);
+                       int32_t tile_m, cudaStream_t st);   // tile_m: 0 = exact importance
 
 // Shared memory the CUDA-core attention kernel needs for a problem, and the most it may ask for.
-size_t simt_attend_smem_bytes(int d, int M, int C, int P, int block_q);
+size_t simt_attend_smem_bytes(int d, int M, int C, int P, int block_q, int tile_m);
 constexpr size_t kSimtAttendSmemLimit = 200 * 1024;
 
 // ---- tensor-core kernels (avq_tc_*.cu) ----

@@ -171,6 +171,8 @@ struct AttendArgs {
   int32_t* topp_out;
   float* importance_out;
   int H, Nq, d, M, C, P, block_q, nblk, stays;
+  int tile_m;     // 0: exact importance; else parents visited in tiles of tile_m (Eq. "aproxdenom")
+  int Nk;
   float scale;
 };
 
@@ -213,6 +215,9 @@ __global__ void __launch_bounds__(kAttendThreads) attend_simt_kernel(AttendArgs 
   float* sbuf = nstay + M;                                         // [nwarps][ncols]
   int* sel = reinterpret_cast<int*>(sbuf + (size_t)nwarps * ncols);   // [M]
   int* sel_list = sel + M;                                         // [max(P,1)]
+  const int ntiles = a.tile_m > 0 ? (M + a.tile_m - 1) / a.tile_m : 0;
+  float* zt = reinterpret_cast<float*>(sel_list + (P > 0 ? P : 1));   // [block_q][ntiles] denominators seen up to a tile
+  float* nseen = zt + (size_t)a.block_q * ntiles;                  // [ntiles] keys of the tiles seen up to a tile
 
   const T* Qb = static_cast<const T*>(a.Q) + ((size_t)bh * a.Nq + i0) * d;
   const T* Cph = static_cast<const T*>(a.Cp) + (size_t)h * M * d;
@@ -246,6 +251,24 @@ __global__ void __launch_bounds__(kAttendThreads) attend_simt_kernel(AttendArgs 
       if (npS[j] > 0.f) z += expf(sb[j] - mx) * npS[j];
     z = warp_sum(z);
     if (lane == 0) { rm[i] = mx; rz[i] = z; }
+    // tiled importance: the part of the denominator contributed by the tiles visited so far
+    float prefix = 0.f;
+    for (int t = 0; t < ntiles; ++t) {
+      float zp = 0.f;
+      const int j1 = min(M, (t + 1) * a.tile_m);
+      for (int j = t * a.tile_m + lane; j < j1; j += 32)
+        if (npS[j] > 0.f) zp += expf(sb[j] - mx) * npS[j];
+      prefix += warp_sum(zp);
+      if (lane == 0) zt[(size_t)i * ntiles + t] = prefix;
+    }
+  }
+  if (tid == 0) {
+    float seen = 0.f;
+    for (int t = 0; t < ntiles; ++t) {
+      const int j1 = min(M, (t + 1) * a.tile_m);
+      for (int j = t * a.tile_m; j < j1; ++j) seen += npS[j];
+      nseen[t] = seen;
+    }
   }
   __syncthreads();
 
@@ -253,11 +276,15 @@ __global__ void __launch_bounds__(kAttendThreads) attend_simt_kernel(AttendArgs 
   for (int j = tid; j < M; j += kAttendThreads) {
     double acc = 0.0;
     if (npS[j] > 0.f) {
+      // exact: the row's full denominator.  Tiled (appendix "Computing Importance with Tiled Codewords"):
+      // the denominator seen up to this codeword's tile, extrapolated by N / N_seen (Eq. "aproxdenom").
+      const int t = ntiles ? j / a.tile_m : 0;
       for (int i = 0; i < rows; ++i) {
         float s = logit(qs + (size_t)i * d, Cph + (size_t)j * d, d, a.scale);
-        acc += (double)expf(s - rm[i]) / (double)rz[i];
+        acc += (double)expf(s - rm[i]) / (double)(ntiles ? zt[(size_t)i * ntiles + t] : rz[i]);
       }
       acc *= (double)npS[j];
+      if (ntiles) acc *= (double)nseen[t] / (double)a.Nk;
     }
     w[j] = acc;
   }
@@ -355,12 +382,13 @@ __global__ void __launch_bounds__(kAttendThreads) attend_simt_kernel(AttendArgs 
 
 }  // namespace (the size below is also used by the host-side validation)
 
-size_t simt_attend_smem_bytes(int d, int M, int C, int P, int block_q) {
+size_t simt_attend_smem_bytes(int d, int M, int C, int P, int block_q, int tile_m) {
   const size_t ncols = (size_t)M + (size_t)P * C;
   size_t b = sizeof(double) * M;
   b += sizeof(float) * ((size_t)block_q * d + 2 * (size_t)block_q + 2 * (size_t)M +
                         (kAttendThreads / 32) * ncols);
   b += sizeof(int) * ((size_t)M + (size_t)(P > 0 ? P : 1));
+  if (tile_m > 0) b += sizeof(float) * ((size_t)block_q + 1) * ((M + tile_m - 1) / tile_m);
   return b;
 }
 
@@ -392,7 +420,7 @@ avq_status launch_aggregate(const avq_problem& p, const void* V, const int32_t* 
 
 template <typename T>
 avq_status launch_attend(const AttendArgs& a, int B, cudaStream_t st) {
-  const size_t smem = simt_attend_smem_bytes(a.d, a.M, a.C, a.P, a.block_q);
+  const size_t smem = simt_attend_smem_bytes(a.d, a.M, a.C, a.P, a.block_q, a.tile_m);
   if (smem > kSimtAttendSmemLimit) return AVQ_ERR_UNSUPPORTED;   // validate_forward rejects these up front
   auto kern = attend_simt_kernel<T>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -427,8 +455,10 @@ avq_status simt_aggregate(const avq_problem& p, const void* V, const int32_t* pa
 avq_status simt_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc,
                        const float* Vp, const float* np_, const float* Vc, const float* nc, int32_t P,
                        int32_t block_q, void* Y, int32_t* topp_out, float* importance_out,
-                       cudaStream_t st) {
+                       int32_t tile_m, cudaStream_t st) {
   AttendArgs a;
+  a.tile_m = tile_m;
+  a.Nk = p.Nk;
   a.Q = Q; a.Cp = Cp; a.Cc = Cc; a.Vp = Vp; a.np_ = np_; a.Vc = Vc; a.nc = nc; a.Y = Y;
   a.topp_out = topp_out; a.importance_out = importance_out;
   a.H = p.H; a.Nq = p.Nq; a.d = p.d; a.M = p.M; a.C = p.C; a.P = P; a.block_q = block_q;
