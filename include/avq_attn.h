@@ -79,7 +79,7 @@ enum {
   /* Algorithm 1's masked scatter: a key moves to its nearest child only if that child is
    * strictly closer than the parent; otherwise it stays with the parent (child index -1).
    * Default (flag clear): every key is represented by the nearest child of its parent.
-   * Supported by the plain CUDA-core kernels only. */
+   * A refined parent then keeps the keys that stayed with it (value sum Vbar_p - sum_c Vbar_c). */
   AVQ_FLAG_PARENT_STAYS = 1u,
   /* Use the plain CUDA-core (FFMA) kernels even where a tensor-core kernel exists.
    * float32 problems always use them.  Meant for cross-checks and for shapes outside the
@@ -103,7 +103,7 @@ typedef struct {
  *     shared memory, 4*block_q*(d + 2) + 20*M + 32*(M + P*C) + 4*max(P, 1) bytes, at most 200 KiB
  *     (e.g. d = 256 with block_q = 256 does not fit; d = 128 with block_q = 256 does).
  *   Tensor-core kernels (bfloat16, no flags): d in {64, 128}; M a multiple of 32, 32..256;
- *     C in {4, 8}; 0 <= P <= M; block_q = 128; scale > 0; AVQ_FLAG_PARENT_STAYS clear.
+ *     C in {4, 8}; 0 <= P <= M; block_q = 128; scale > 0.
  */
 
 /* Bytes of device scratch avq_forward needs for this problem (0 if the problem is invalid).

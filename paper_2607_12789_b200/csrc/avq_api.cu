@@ -27,7 +27,6 @@ avq_status validate_problem(const avq_problem* p) {
   if ((int64_t)p->B * p->H * (int64_t)(p->Nq > p->Nk ? p->Nq : p->Nk) * p->d >= ((int64_t)1 << 40))
     return AVQ_ERR_UNSUPPORTED;
   if (use_tensor_path(*p)) {
-    if (p->flags & AVQ_FLAG_PARENT_STAYS) return AVQ_ERR_UNSUPPORTED;
     if (p->d != 64 && p->d != 128) return AVQ_ERR_UNSUPPORTED;
     if (p->M % 32 != 0 || p->M < 32 || p->M > 256) return AVQ_ERR_UNSUPPORTED;
     if (p->C != 4 && p->C != 8) return AVQ_ERR_UNSUPPORTED;
@@ -69,6 +68,10 @@ Layout make_layout(const avq_problem& p, int32_t /*P*/, int32_t /*block_q*/) {
   if (use_tensor_path(p)) {
     L.Vpb = take(2 * BH * p.M * p.d);
     L.Vcb = take(2 * BH * p.M * p.C * p.d);
+    if (p.flags & AVQ_FLAG_PARENT_STAYS) {
+      L.Vsb = take(2 * BH * p.M * p.d);
+      L.rho = take(sizeof(float) * BH * p.M);
+    }
   }
   L.total = off;
   return L;
@@ -123,7 +126,7 @@ avq_status avq_aggregate(const avq_problem* prob, const void* V, const int32_t* 
     return AVQ_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (use_tensor_path(*prob))
-    return tc_aggregate(*prob, V, parent_idx, child_idx, Vp, np_, Vc, nc, nullptr, nullptr, false, nullptr, st);
+    return tc_aggregate(*prob, V, parent_idx, child_idx, Vp, np_, Vc, nc, nullptr, nullptr, nullptr, nullptr, false, nullptr, st);
   return simt_aggregate(*prob, V, parent_idx, child_idx, Vp, np_, Vc, nc, st);
 }
 
@@ -131,7 +134,8 @@ namespace {
 struct Regions {
   int32_t *status_word, *pidx, *cidx;
   float *Vp, *np_, *Vc, *nc;
-  void *Vpb, *Vcb;
+  void *Vpb, *Vcb, *Vsb;
+  float* rho;
 };
 Regions carve(void* workspace, const Layout& L) {
   char* ws = static_cast<char*>(workspace);
@@ -145,13 +149,15 @@ Regions carve(void* workspace, const Layout& L) {
   r.nc = reinterpret_cast<float*>(ws + L.nc);
   r.Vpb = ws + L.Vpb;
   r.Vcb = ws + L.Vcb;
+  r.Vsb = L.Vsb ? ws + L.Vsb : nullptr;
+  r.rho = L.rho ? reinterpret_cast<float*>(ws + L.rho) : nullptr;
   return r;
 }
 avq_status attend_stage(const avq_problem& p, const Regions& r, const void* Q, const void* Cp, const void* Cc,
                         int32_t P, int32_t block_q, void* Y, int32_t* topp_out, float* importance_out,
                         bool chained, cudaStream_t st) {
   if (use_tensor_path(p))
-    return tc_attend(p, Q, Cp, Cc, r.np_, r.nc, r.Vpb, r.Vcb, P, Y, topp_out, importance_out, r.status_word,
+    return tc_attend(p, Q, Cp, Cc, r.np_, r.nc, r.Vpb, r.Vcb, r.Vsb, r.rho, P, Y, topp_out, importance_out, r.status_word,
                      chained, st);
   return simt_attend(p, Q, Cp, Cc, r.Vp, r.np_, r.Vc, r.nc, P, block_q, Y, topp_out, importance_out, 0, st);
 }
@@ -185,7 +191,7 @@ avq_status avq_forward(const avq_problem* prob, const void* Q, const void* K, co
     // status header, leaf sums and leaf counts are adjacent: the assign grid clears them on the side
     s = tc_assign(p, K, Cp, Cc, r.pidx, r.cidx, r.status_word, workspace, L.zero_end, st);
     if (s != AVQ_OK) return s;
-    s = tc_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, r.Vpb, r.Vcb, true, r.status_word, st);
+    s = tc_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, r.Vpb, r.Vcb, r.Vsb, r.rho, true, r.status_word, st);
   } else {
     if (cudaMemsetAsync(r.status_word, 0, 256, st) != cudaSuccess) return AVQ_ERR_CUDA;
     s = simt_assign(p, K, Cp, Cc, r.pidx, r.cidx, st);

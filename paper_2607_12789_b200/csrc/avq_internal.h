@@ -21,6 +21,8 @@ struct Layout {
   size_t child_idx = 0;    // int32 [B,H,Nk]
   size_t Vpb = 0;          // bf16 [B,H,M,d]      copy of Vp (tensor-core path only)
   size_t Vcb = 0;          // bf16 [B,H,M,C,d]    copy of Vc (tensor-core path only)
+  size_t Vsb = 0;          // bf16 [B,H,M,d]      stay residual rows (tensor-core path, PARENT_STAYS)
+  size_t rho = 0;          // f32 [B,H,M]         share of a parent's keys that stay
   size_t total = 0;
 };
 
@@ -60,9 +62,11 @@ avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const 
                      size_t zero_bytes, cudaStream_t st);
 avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
                         const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc,
-                        void* Vpb, void* Vcb, bool pre_zeroed, int32_t* status_word, cudaStream_t st);
+                        void* Vpb, void* Vcb, void* Vsb, float* rho, bool pre_zeroed, int32_t* status_word,
+                        cudaStream_t st);   // Vsb, rho: stay rows and stay shares (PARENT_STAYS), may be null
 avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc,
-                     const float* np_, const float* nc, const void* Vpb, const void* Vcb, int32_t P,
+                     const float* np_, const float* nc, const void* Vpb, const void* Vcb, const void* Vsb,
+                     const float* rho, int32_t P,
                      void* Y, int32_t* topp_out, float* importance_out, int32_t* status_word,
                      bool chained, cudaStream_t st);   // chained: launched right behind tc_aggregate
 

@@ -236,7 +236,7 @@ template <int D, int C>
 __global__ void __launch_bounds__(D)
 finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, float* __restrict__ Vp,
                 float* __restrict__ np_, __nv_bfloat16* __restrict__ Vpb, __nv_bfloat16* __restrict__ Vcb,
-                int M, const int32_t* status_word) {
+                __nv_bfloat16* __restrict__ Vsb, float* __restrict__ rho, int M, const int32_t* status_word) {
   tc::pdl_launch_dependents();
   tc::pdl_wait();                                    // the leaf sums come from the kernel before
   if (status_word && *reinterpret_cast<const volatile int32_t*>(status_word) != 0) return;
@@ -269,7 +269,12 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
         if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(cn[mm][c] > 0.f ? x[mm][c] * __frcp_rn(cn[mm][c]) : 0.f);
       }
       Vp[row * D + k] = s;
-      if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(n > 0.f ? s * __frcp_rn(n) : 0.f);
+      const float rn = n > 0.f ? __frcp_rn(n) : 0.f;
+      if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(s * rn);
+      // what a refined parent keeps under the PARENT_STAYS rule, per key of the parent: its weight in the
+      // attention kernel is A n_p, so the row is Vbar_stay / n_p and the count n_stay / n_p
+      if (Vsb) Vsb[row * D + k] = __float2bfloat16_rn(stay[mm] * rn);
+      if (rho && k == 0) rho[row] = nstay[mm] * rn;
     }
   }
   __syncthreads();                                     // every thread has read the stay counts
@@ -284,8 +289,8 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
 
 template <int D, int C>
 avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const int32_t* cidx, float* Vp,
-               float* np_, float* Vc, float* nc, void* Vpb, void* Vcb, bool pre_zeroed, int32_t* status_word,
-               cudaStream_t st) {
+               float* np_, float* Vc, float* nc, void* Vpb, void* Vcb, void* Vsb, float* rho, bool pre_zeroed,
+               int32_t* status_word, cudaStream_t st) {
   const unsigned BH = (unsigned)(p.B * p.H);
   if (!pre_zeroed) {
     if (cudaMemsetAsync(Vc, 0, sizeof(float) * (size_t)BH * p.M * C * D, st) != cudaSuccess) return AVQ_ERR_CUDA;
@@ -341,19 +346,20 @@ avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const i
   dim3 g2(p.M / 8, BH);
   return cuda_ok(tc::launch_pdl(finalize_kernel<D, C>, g2, dim3(D), 0, st, true, static_cast<const float*>(Vc),
                                 static_cast<const float*>(nc), Vp, np_, static_cast<__nv_bfloat16*>(Vpb),
-                                static_cast<__nv_bfloat16*>(Vcb), p.M, static_cast<const int32_t*>(status_word)));
+                                static_cast<__nv_bfloat16*>(Vcb), static_cast<__nv_bfloat16*>(Vsb), rho, p.M,
+                                static_cast<const int32_t*>(status_word)));
 }
 
 }  // namespace
 
 avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
                         const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc, void* Vpb,
-                        void* Vcb, bool pre_zeroed, int32_t* status_word, cudaStream_t st) {
+                        void* Vcb, void* Vsb, float* rho, bool pre_zeroed, int32_t* status_word, cudaStream_t st) {
   if (p.d == 64)
-    return p.C == 4 ? run<64, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, status_word, st)
-                    : run<64, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, status_word, st);
-  return p.C == 4 ? run<128, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, status_word, st)
-                  : run<128, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, pre_zeroed, status_word, st);
+    return p.C == 4 ? run<64, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, Vsb, rho, pre_zeroed, status_word, st)
+                    : run<64, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, Vsb, rho, pre_zeroed, status_word, st);
+  return p.C == 4 ? run<128, 4>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, Vsb, rho, pre_zeroed, status_word, st)
+                  : run<128, 8>(p, V, parent_idx, child_idx, Vp, np_, Vc, nc, Vpb, Vcb, Vsb, rho, pre_zeroed, status_word, st);
 }
 
 }  // namespace avq

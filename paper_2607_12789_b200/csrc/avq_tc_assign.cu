@@ -73,7 +73,9 @@ __device__ double exact_dist_smem(const unsigned char* Ks, int row, const __nv_b
 }
 
 // NL = 16-byte loads per lane that cover one parent's C x d block of children: C * d / 256.
-template <int D, int NL>
+// STAYS: Algorithm 1's masked scatter - a key moves to its nearest child only if that child is strictly
+// closer than the parent (child index -1 otherwise).
+template <int D, int NL, bool STAYS>
 __global__ void __launch_bounds__(kThreadsA, assign_min_ctas(D, NL))
 tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmCp,
                  const __nv_bfloat16* __restrict__ Cp, const __nv_bfloat16* __restrict__ Cc,
@@ -261,6 +263,7 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       for (int c = 0; c < kC; ++c) dst[c] = __ldg(src + c * kChunks);
     };
     float sum[kC];
+    float sum_p = 0.f;                                   // STAYS: direct-form distance to the parent itself
     issue(0, buf[0]);
   #pragma unroll
     for (int step = 0; step < kSteps; ++step) {
@@ -270,11 +273,14 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       if (t == 0) {
   #pragma unroll
         for (int c = 0; c < kC; ++c) sum[c] = 0.f;
+        sum_p = 0.f;
       }
       const int ch = s4 + 4 * t;
       const KeyChunk kv = widen8(*reinterpret_cast<const uint4*>(Ks + (ch >> 3) * (kKeys * 128) + sw128_offset(key, (ch & 7) * 8)));
   #pragma unroll
       for (int c = 0; c < kC; ++c) sum[c] += sqdiff8(kv, buf[step & 1][c]);
+      if constexpr (STAYS)
+        sum_p += sqdiff8(kv, __ldg(reinterpret_cast<const uint4*>(Cp + (head_base + par[key]) * D) + ch));
       if (t == kT - 1) {
         // transpose-reduce over the group: after the two exchanges lane s holds the total of child s
         // (and of child s + 4 when C = 8)
@@ -307,16 +313,32 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
           e2 = fminf(fmaxf(e1, b1), fminf(e2, b2));
           if (b1 < e1 || (b1 == e1 && cb < c1)) { e1 = b1; c1 = cb; }
         }
+        float dp = 0.f;
+        if constexpr (STAYS) {
+          dp = sum_p + __shfl_xor_sync(0xffffffffu, sum_p, 1);
+          dp += __shfl_xor_sync(0xffffffffu, dp, 2);
+        }
         if (s4 == 0) {
+          bool rechecked = false;
+          double best = INFINITY;
           if (done && j0 + key < Nk && !(e2 - e1 > 1e-4f * e2)) {
             const __nv_bfloat16* Cch = Cc + (head_base + par[key]) * kC * D;
-            double best = INFINITY;
             int bi = 0;
             for (int c = 0; c < kC; ++c) {
               const double sd = exact_dist_smem<D>(Ks, key, Cch + (size_t)c * D);
               if (sd < best) { best = sd; bi = c; }
             }
             c1 = bi;
+            rechecked = true;
+          }
+          if constexpr (STAYS) {
+            // strict '<' against the parent distance; float64 when the two are closer than fp32 separates
+            bool moved = e1 < dp;
+            if (done && j0 + key < Nk && (rechecked || !(fabsf(e1 - dp) > 1e-4f * fmaxf(e1, dp)))) {
+              if (!rechecked) best = exact_dist_smem<D>(Ks, key, Cc + ((head_base + par[key]) * kC + c1) * D);
+              moved = best < exact_dist_smem<D>(Ks, key, Cp + (head_base + par[key]) * D);
+            }
+            if (!moved) c1 = -1;
           }
           chi[key] = c1;
         }
@@ -339,7 +361,7 @@ uint32_t pow2_cols(int n) {
   return c;
 }
 
-template <int D, int NL>
+template <int D, int NL, bool STAYS>
 avq_status launch(const avq_problem& p, const void* K, const void* Cp, const void* Cc, int32_t* pidx,
                   int32_t* cidx, int32_t* status_word, void* zero_base, size_t zero_bytes, cudaStream_t st) {
   CUtensorMap tmK, tmCp;
@@ -359,7 +381,7 @@ avq_status launch(const avq_problem& p, const void* K, const void* Cp, const voi
   const size_t smem = (size_t)(D / 64) * (kKeys + p.M) * 128 +
                       sizeof(float) * (p.M + 6 * kKeys) +
                       sizeof(int) * (4 * kKeys) + 64 + 1024;
-  auto kern = tc_assign_kernel<D, NL>;
+  auto kern = tc_assign_kernel<D, NL, STAYS>;
   // The limit is set once per device and instantiation (setting it again is harmless if two threads race).
   static size_t configured[64] = {};
   int dev = 0;
@@ -383,11 +405,13 @@ avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const 
                      int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, void* zero_base,
                      size_t zero_bytes, cudaStream_t st) {
   if (zero_bytes % 16 != 0 || (zero_bytes / 16) >> 31) return AVQ_ERR_WORKSPACE;
-  if (p.d == 64)
-    return p.C == 4 ? launch<64, 1>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st)
-                    : launch<64, 2>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st);
-  return p.C == 4 ? launch<128, 2>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st)
-                  : launch<128, 4>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st);
+  const bool stays = (p.flags & AVQ_FLAG_PARENT_STAYS) != 0;
+#define AVQ_ASSIGN(DD, NN)                                                                                     \
+  (stays ? launch<DD, NN, true>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st) \
+         : launch<DD, NN, false>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st))
+  if (p.d == 64) return p.C == 4 ? AVQ_ASSIGN(64, 1) : AVQ_ASSIGN(64, 2);
+  return p.C == 4 ? AVQ_ASSIGN(128, 2) : AVQ_ASSIGN(128, 4);
+#undef AVQ_ASSIGN
 }
 
 }  // namespace avq

@@ -30,6 +30,8 @@ constexpr int kRows = 128;
 struct AttendParams {
   const __nv_bfloat16* Cc;    // [H, M, C, d]
   const __nv_bfloat16* Vcb;   // [B*H, M, C, d]
+  const __nv_bfloat16* Vsb;   // [B*H, M, d]  PARENT_STAYS: value sum of the keys that stay / all keys of the parent
+  const float* rho;           // [B*H, M]     PARENT_STAYS: keys that stay / all keys of the parent (else nullptr)
   const float* np_;           // [B*H, M]
   const float* nc;            // [B*H, M, C]
   __nv_bfloat16* Y;           // [B*H, Nq, d]
@@ -455,7 +457,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       int pos = __popc(bal & ((1u << lane) - 1u));
       for (int u = 0; u < warp; ++u) pos += __popc(wmask[u]);
       sel_list[pos] = j;
-      cntk[j] = 0.f;
+      cntk[j] = p.rho ? __ldg(p.rho + (size_t)bh * M + j) : 0.f;   // the share of its keys that stays with it
       if (p.topp_out) p.topp_out[((size_t)bh * p.nblk + blk) * P + pos] = j;
     }
   }
@@ -514,7 +516,12 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   mbar_wait(bar_ld1, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);   // value sums have landed
   for (int u = tid; u < (min(P, M) << kLogChunks); u += kThreads) {
     const int row = sel_list[u >> kLogChunks], ch = u & ((1 << kLogChunks) - 1);
-    *reinterpret_cast<uint4*>(Vs + (ch >> 3) * (M * 128) + sw128_offset(row, (ch & 7) * 8)) = make_uint4(0, 0, 0, 0);
+    // a refined parent keeps only the keys that stayed with it (Algorithm 1's masked scatter): its value row
+    // becomes the stay residual, Vbar_stay = Vbar_p - sum_c Vbar_c, in the same per-n_p units (all zero under
+    // the default rule, where every key moves to a child)
+    uint4 stay = make_uint4(0, 0, 0, 0);
+    if (p.Vsb) stay = __ldg(reinterpret_cast<const uint4*>(p.Vsb + ((size_t)bh * M + row) * D) + ch);
+    *reinterpret_cast<uint4*>(Vs + (ch >> 3) * (M * 128) + sw128_offset(row, (ch & 7) * 8)) = stay;
   }
   {
     float zloc = 0.f;
@@ -750,7 +757,7 @@ avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUte
 
 template <int D>
 avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const void* Cc, const float* np_,
-                  const float* nc, const void* Vpb, const void* Vcb, int32_t P, void* Y, int32_t* topp_out,
+                  const float* nc, const void* Vpb, const void* Vcb, const void* Vsb, const float* rho, int32_t P, void* Y, int32_t* topp_out,
                   float* importance_out, int32_t* status_word, bool chained, cudaStream_t st) {
   const uint64_t BH = (uint64_t)p.B * p.H;
   CUtensorMap tmQ, tmCp, tmVpb, tmY;
@@ -777,6 +784,8 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
   AttendParams a;
   a.Cc = static_cast<const __nv_bfloat16*>(Cc);
   a.Vcb = static_cast<const __nv_bfloat16*>(Vcb);
+  a.Vsb = static_cast<const __nv_bfloat16*>(Vsb);
+  a.rho = rho;
   a.np_ = np_;
   a.nc = nc;
   a.Y = static_cast<__nv_bfloat16*>(Y);
@@ -812,10 +821,10 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
 }  // namespace
 
 avq_status tc_attend(const avq_problem& p, const void* Q, const void* Cp, const void* Cc, const float* np_,
-                     const float* nc, const void* Vpb, const void* Vcb, int32_t P, void* Y, int32_t* topp_out,
+                     const float* nc, const void* Vpb, const void* Vcb, const void* Vsb, const float* rho, int32_t P, void* Y, int32_t* topp_out,
                      float* importance_out, int32_t* status_word, bool chained, cudaStream_t st) {
-  return p.d == 64 ? launch<64>(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, P, Y, topp_out, importance_out, status_word, chained, st)
-                   : launch<128>(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, P, Y, topp_out, importance_out, status_word, chained, st);
+  return p.d == 64 ? launch<64>(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, Vsb, rho, P, Y, topp_out, importance_out, status_word, chained, st)
+                   : launch<128>(p, Q, Cp, Cc, np_, nc, Vpb, Vcb, Vsb, rho, P, Y, topp_out, importance_out, status_word, chained, st);
 }
 
 }  // namespace avq

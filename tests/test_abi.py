@@ -61,7 +61,6 @@ def test_workspace_bytes_and_layout(lib):
     (dict(d=256), 2, 256, 3),                                   # CUDA-core attention tile beyond 200 KiB of shared memory
     (dict(dtype_code=binding.AVQ_BF16, d=96), 2, 128, 3), (dict(dtype_code=binding.AVQ_BF16, M=24), 2, 128, 3),
     (dict(dtype_code=binding.AVQ_BF16, C=3), 2, 128, 3), (dict(dtype_code=binding.AVQ_BF16), 2, 64, 3),
-    (dict(dtype_code=binding.AVQ_BF16, flags=binding.FLAG_PARENT_STAYS), 2, 128, 3),
 ])
 def test_invalid_problems_are_rejected_on_the_host(lib, kw, P, bq, want):
     p = _prob(**kw)

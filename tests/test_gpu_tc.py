@@ -122,6 +122,29 @@ def test_other_shapes_d128_C8_M96():
                                       alpha=0.5, hot_queries=True))
 
 
+@pytest.mark.parametrize("wl", [synth.C1.with_(B=2, H=2, N=1500, seed=51), synth.C3.with_(H=2, N=2000, seed=52),
+                                synth.C2.with_(B=1, H=2, N=1100, seed=53)],
+                         ids=["d64_M64_C4", "d128_M256_C4", "d64_M128_C8"])
+def test_parent_stays_on_the_tensor_core_path(wl):
+    """Algorithm 1's masked scatter on the tcgen05 path: half of the keys hug their parent and stay with it
+    (child index -1), the others move to a child; a refined parent keeps the stay residual."""
+    x = synth.generate(wl)
+    g = np.random.default_rng(wl.seed)
+    for b in range(wl.B):
+        for h in range(wl.H):
+            near = x["Cp"][h][g.integers(0, wl.M, wl.N // 2)] + 0.05 * g.standard_normal((wl.N // 2, wl.d))
+            x["K"][b, h, ::2] = synth.round_to_bf16(near.astype(np.float32))[: len(x["K"][b, h, ::2])]
+    rep = parity.full_parity(wl, flags=binding.FLAG_PARENT_STAYS, parent_stays=True, x=x)
+    print("stays", rep)
+    total = wl.B * wl.H * wl.N
+    assert 0.3 * total <= rep["stay_count"] <= 0.7 * total        # a real mixture of stayed and moved keys
+    # and the two rules really differ on this input
+    gpu_rep = parity.gpu_forward(wl, x, flags=0)
+    gpu_st = parity.gpu_forward(wl, x, flags=binding.FLAG_PARENT_STAYS)
+    assert (gpu_rep["child_idx"] >= 0).all() and (gpu_st["child_idx"] < 0).any()
+    assert np.abs(gpu_rep["Y"] - gpu_st["Y"]).max() > 1e-3
+
+
 def test_tensor_core_and_cuda_core_paths_agree_at_full_size():
     wl = synth.C3.with_(H=4)
     dv = parity.to_device(synth.generate(wl), "bf16")
