@@ -84,7 +84,13 @@ enum {
   /* Use the plain CUDA-core (FFMA) kernels even where a tensor-core kernel exists.
    * float32 problems always use them.  Meant for cross-checks and for shapes outside the
    * tensor-core envelope. */
-  AVQ_FLAG_SIMT = 2u
+  AVQ_FLAG_SIMT = 2u,
+  /* Algorithm 2's child pass as printed: the parent's logit is recovered as the mean of its children's
+   * logits (Eq. "parent_recovery") and the children add the differences Delta A = A_c - A_p to accumulators
+   * that keep every parent's full term (Eq. "correcting_attention").  Equal to the default (masked) form only
+   * for codebooks that satisfy parent = mean(children); CUDA-core kernels only (with bfloat16 inputs set
+   * AVQ_FLAG_SIMT too: rounding the codebook to bfloat16 already breaks the constraint by an ulp). */
+  AVQ_FLAG_CORRECTING = 4u
 };
 
 typedef struct {

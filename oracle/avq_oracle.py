@@ -21,6 +21,8 @@ What each function follows in the paper:
                          a key is represented by its child codeword if its parent was
                          selected for that block (and the key moved to a child), else by
                          its parent codeword ("quantised-key attention", Sec. 3.2).
+* ``forward_block_correcting`` - Algorithm 2's child pass as printed (mean-recovered parent logit,
+                         Eq. "parent_recovery"; Delta A updates, Eq. "correcting_attention").
 * ``forward_block_factorised`` - the O(M N) regrouped form of the same quantity
                          (Sec. 3.2 regrouping + the post-refinement sum of the appendix
                          "Correcting Attention Derivation": ``A_p Vbar_stay + sum_c A_c Vbar_c``).
@@ -308,6 +310,32 @@ def forward_block_factorised(Qb, Cp, Cc, Vp, n_p, Vc, n_c, selected, scale: floa
     return (A @ vals) / (A @ cnts)[:, None]
 
 
+def forward_block_correcting(Qb, Cp, Cc, Vp, n_p, Vc, n_c, selected, scale: float):
+    """Algorithm 2's child pass as printed: every parent keeps its full term ``e^{s_p} (Vp_p, n_p)``; for a
+    selected parent the logit is RECOVERED as the mean of its children's logits (Eq. "parent_recovery") and
+    each non-empty child adds ``(e^{s_pc} - e^{s_p,rec}) (Vc_pc, n_pc)`` (Eq. "correcting_attention").
+    Equals ``forward_block_factorised`` when every parent is the mean of its children."""
+    Qb = np.asarray(Qb, dtype=F64)
+    Cp = np.asarray(Cp, dtype=F64)
+    Cc = np.asarray(Cc, dtype=F64)
+    selected = np.asarray(selected, dtype=np.int64)
+    s_p = scale * (Qb @ Cp.T)                                     # [bq, M]
+    s_c = scale * np.einsum("id,pcd->ipc", Qb, Cc[selected])      # [bq, P, C]
+    s_rec = s_c.mean(axis=2)                                      # recovered parent logits
+    live_p = n_p > 0
+    live_c = n_c[selected] > 0
+    m = np.max(np.where(live_p[None, :], s_p, -np.inf), axis=1)
+    if selected.size:
+        m = np.maximum(m, np.max(np.where(live_c[None], s_c, -np.inf), axis=(1, 2)))
+    A_p = np.where(live_p[None, :], np.exp(s_p - m[:, None]), 0.0)
+    X = A_p @ Vp
+    Z = A_p @ n_p
+    dA = np.where(live_c[None], np.exp(s_c - m[:, None, None]) - np.exp(s_rec - m[:, None])[:, :, None], 0.0)
+    X = X + np.einsum("ipc,pcd->id", dA, Vc[selected])
+    Z = Z + np.einsum("ipc,pc->i", dA, n_c[selected])
+    return X / Z[:, None]
+
+
 # --------------------------------------------------------------------------- forward, one head / all heads
 def forward_head(Q, K, V, Cp, Cc, P: int, block_q: int, scale: float, parent_stays: bool = False,
                  form: str = "dense", blocks=None, assignment=None, tile_m: int | None = None):
@@ -353,6 +381,8 @@ def forward_head(Q, K, V, Cp, Cc, P: int, block_q: int, scale: float, parent_sta
             Y[i0:i1] = forward_block_dense(Qb, V, Cp64, Cc64, pidx, cidx, sel, scale)
         elif form == "factorised":
             Y[i0:i1] = forward_block_factorised(Qb, Cp64, Cc64, Vp, n_p, Vc, n_c, sel, scale)
+        elif form == "correcting":
+            Y[i0:i1] = forward_block_correcting(Qb, Cp64, Cc64, Vp, n_p, Vc, n_c, sel, scale)
         else:
             raise ValueError(form)
     return dict(Y=Y, selected=selected, importance=importance, topp_margin=margins, assignment=asg,

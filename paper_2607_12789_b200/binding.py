@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "lib", "libavq_attn.so")
 
 AVQ_F32, AVQ_BF16 = 0, 1
-FLAG_PARENT_STAYS, FLAG_SIMT = 1, 2
+FLAG_PARENT_STAYS, FLAG_SIMT, FLAG_CORRECTING = 1, 2, 4
 STATUS_NAMES = {0: "AVQ_OK", 1: "AVQ_ERR_NULL", 2: "AVQ_ERR_SHAPE", 3: "AVQ_ERR_UNSUPPORTED", 4: "AVQ_ERR_ALIGN",
                 5: "AVQ_ERR_WORKSPACE", 6: "AVQ_ERR_CUDA", 7: "AVQ_ERR_DEVICE_TIMEOUT", 8: "AVQ_ERR_INDEX"}
 

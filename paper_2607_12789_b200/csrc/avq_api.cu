@@ -22,11 +22,12 @@ avq_status validate_problem(const avq_problem* p) {
     return AVQ_ERR_SHAPE;
   if (p->dtype != AVQ_F32 && p->dtype != AVQ_BF16) return AVQ_ERR_SHAPE;
   if (!isfinite(p->scale)) return AVQ_ERR_SHAPE;
-  if (p->flags & ~(uint32_t)(AVQ_FLAG_PARENT_STAYS | AVQ_FLAG_SIMT)) return AVQ_ERR_SHAPE;
+  if (p->flags & ~(uint32_t)(AVQ_FLAG_PARENT_STAYS | AVQ_FLAG_SIMT | AVQ_FLAG_CORRECTING)) return AVQ_ERR_SHAPE;
   if ((int64_t)p->B * p->H > 65535) return AVQ_ERR_UNSUPPORTED;
   if ((int64_t)p->B * p->H * (int64_t)(p->Nq > p->Nk ? p->Nq : p->Nk) * p->d >= ((int64_t)1 << 40))
     return AVQ_ERR_UNSUPPORTED;
   if (use_tensor_path(*p)) {
+    if (p->flags & AVQ_FLAG_CORRECTING) return AVQ_ERR_UNSUPPORTED;   // the tensor-core kernel is the masked form
     if (p->d != 64 && p->d != 128) return AVQ_ERR_UNSUPPORTED;
     if (p->M % 32 != 0 || p->M < 32 || p->M > 256) return AVQ_ERR_UNSUPPORTED;
     if (p->C != 4 && p->C != 8) return AVQ_ERR_UNSUPPORTED;

@@ -171,6 +171,7 @@ struct AttendArgs {
   int32_t* topp_out;
   float* importance_out;
   int H, Nq, d, M, C, P, block_q, nblk, stays;
+  int correcting; // Algorithm 2's literal child pass: mean-recovered parent logit and Delta A = A_c - A_p
   int tile_m;     // 0: exact importance; else parents visited in tiles of tile_m (Eq. "aproxdenom")
   int Nk;
   float scale;
@@ -326,7 +327,7 @@ __global__ void __launch_bounds__(kAttendThreads) attend_simt_kernel(AttendArgs 
     for (int j = lane; j < M; j += 32) {
       float s = logit(q, Cph + (size_t)j * d, d, a.scale);
       sb[j] = s;
-      const float cnt = sel[j] ? (a.stays ? nstay[j] : 0.f) : npS[j];
+      const float cnt = (sel[j] && !a.correcting) ? (a.stays ? nstay[j] : 0.f) : npS[j];
       if (cnt > 0.f) mx = fmaxf(mx, s);
     }
     for (int e = lane; e < P * C; e += 32) {
@@ -342,7 +343,8 @@ __global__ void __launch_bounds__(kAttendThreads) attend_simt_kernel(AttendArgs 
     for (int u = 0; u < kMaxDPerLane; ++u) x[u] = 0.f;
     float z = 0.f;
     for (int j = 0; j < M; ++j) {
-      const bool s_ = sel[j] != 0;
+      // correcting form: every parent keeps its full term here, the children add differences below
+      const bool s_ = sel[j] != 0 && !a.correcting;
       const float cnt = s_ ? (a.stays ? nstay[j] : 0.f) : npS[j];
       if (!(cnt > 0.f)) continue;
       const float av = expf(sb[j] - mx);
@@ -362,7 +364,14 @@ __global__ void __launch_bounds__(kAttendThreads) attend_simt_kernel(AttendArgs 
       const int p = sel_list[e / C], c = e % C;
       const float cnt = nc[p * C + c];
       if (!(cnt > 0.f)) continue;
-      const float av = expf(sb[M + e] - mx);
+      float av = expf(sb[M + e] - mx);
+      if (a.correcting) {
+        // Eq. "parent_recovery": under parent = mean(children) the parent's logit is the mean of its
+        // children's; Eq. "correcting_attention": the child's keys trade the parent's weight for their own
+        float sp = 0.f;
+        for (int c2 = 0; c2 < C; ++c2) sp += sb[M + (e / C) * C + c2];
+        av -= expf(sp / (float)C - mx);
+      }
       z += av * cnt;
 #pragma unroll
       for (int u = 0; u < kMaxDPerLane; ++u) {
@@ -464,6 +473,7 @@ avq_status simt_attend(const avq_problem& p, const void* Q, const void* Cp, cons
   a.H = p.H; a.Nq = p.Nq; a.d = p.d; a.M = p.M; a.C = p.C; a.P = P; a.block_q = block_q;
   a.nblk = (p.Nq + block_q - 1) / block_q;
   a.stays = (p.flags & AVQ_FLAG_PARENT_STAYS) ? 1 : 0;
+  a.correcting = (p.flags & AVQ_FLAG_CORRECTING) ? 1 : 0;
   a.scale = p.scale;
   return p.dtype == AVQ_F32 ? launch_attend<float>(a, p.B, st) : launch_attend<__nv_bfloat16>(a, p.B, st);
 }

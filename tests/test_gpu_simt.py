@@ -93,3 +93,31 @@ def test_forward_host_matches_device_call():
     torch.cuda.synchronize()
     f.check()
     assert torch.allclose(hy, Y.cpu(), atol=1e-6)
+
+
+def test_correcting_form_matches_the_oracle_and_the_masked_form_on_recentred_codebooks():
+    """AVQ_FLAG_CORRECTING (Algorithm 2's child pass as printed) on the CUDA-core kernels.  float32, re-centred
+    children: equal to the oracle's correcting form and (the constraint holds to fp32 rounding) to the default
+    masked form.  bfloat16 codebooks: rounding breaks parent = mean(children) by an ulp, so the kernel is
+    compared with the oracle's correcting form on the same rounded codebooks, and its distance from the masked
+    form is what the variant costs in accuracy."""
+    wl = synth.C0.with_(H=2, seed=33, recenter_children=True)
+    x = synth.generate(wl)
+    dv = parity.to_device(x, "f32")
+    args = (dv["Q"], dv["K"], dv["V"], dv["Cp"], dv["Cc"], wl.P, wl.block_q)
+    Yc = binding.forward(*args, scale=wl.scale, flags=binding.FLAG_CORRECTING)
+    Ym = binding.forward(*args, scale=wl.scale)
+    ref = orc.forward(x["Q"], x["K"], x["V"], x["Cp"], x["Cc"], wl.P, wl.block_q, wl.scale, form="correcting")
+    assert np.abs(Yc.cpu().numpy() - ref["Y"]).max() <= 1e-4
+    assert (Yc - Ym).abs().max().item() <= 1e-4
+    wl = synth.C1.with_(B=1, H=2, N=512, seed=34, recenter_children=True)
+    x = synth.generate(wl)
+    dv = parity.to_device(x, "bf16")
+    args = (dv["Q"], dv["K"], dv["V"], dv["Cp"], dv["Cc"], wl.P, wl.block_q)
+    Yc = binding.forward(*args, scale=wl.scale, flags=binding.FLAG_CORRECTING | SIMT)
+    Ym = binding.forward(*args, scale=wl.scale, flags=SIMT)
+    ref = orc.forward(x["Q"], x["K"], x["V"], x["Cp"], x["Cc"], wl.P, wl.block_q, wl.scale, form="correcting")
+    assert np.abs(Yc.float().cpu().numpy() - ref["Y"]).max() <= 2e-2
+    dev = (Yc.float() - Ym.float()).abs().max().item()
+    print(f"correcting vs masked form, bf16-rounded re-centred codebooks: max-abs {dev:.3e}")
+    assert dev <= 0.25

@@ -275,3 +275,25 @@ def test_benchmark_generator_structure():
         assert np.array_equal(synth.round_to_bf16(v), v), k          # already bf16-representable
     y = synth.generate(synth.C1.with_(B=1, H=2))
     assert all(np.array_equal(x[k], y[k]) for k in x)                 # seeded, reproducible
+
+
+@pytest.mark.parametrize("parent_stays", [False, True])
+def test_correcting_form_equals_the_definition_exactly_when_parents_are_child_means(parent_stays):
+    """Algorithm 2 as printed (mean-recovered logit, Delta A) against the dense definition: equal on codebooks
+    that satisfy parent = mean(children) in float64, visibly different on codebooks that do not."""
+    g = np.random.default_rng(17)
+    M, C, d, N = 10, 3, 5, 150
+    Cp = g.normal(size=(M, d)) * 2
+    Cc = Cp[:, None, :] + 0.5 * g.normal(size=(M, C, d))
+    Cc_ok = Cc - Cc.mean(axis=1, keepdims=True) + Cp[:, None, :]
+    K = np.concatenate([Cc_ok[g.integers(0, M, N // 2), g.integers(0, C, N // 2)] + 0.2 * g.normal(size=(N // 2, d)),
+                        Cp[g.integers(0, M, N - N // 2)] + 0.05 * g.normal(size=(N - N // 2, d))])
+    Q, V = g.normal(size=(N, d)), g.normal(size=(N, d))
+    dense = orc.forward_head(Q, K, V, Cp, Cc_ok, 4, 50, 0.6, parent_stays=parent_stays, form="dense")
+    corr = orc.forward_head(Q, K, V, Cp, Cc_ok, 4, 50, 0.6, parent_stays=parent_stays, form="correcting")
+    np.testing.assert_allclose(corr["Y"], dense["Y"], atol=1e-12)
+    if parent_stays:
+        assert (dense["assignment"]["child_idx"] < 0).any()
+    bad = orc.forward_head(Q, K, V, Cp, Cc, 4, 50, 0.6, parent_stays=parent_stays, form="correcting")
+    good = orc.forward_head(Q, K, V, Cp, Cc, 4, 50, 0.6, parent_stays=parent_stays, form="dense")
+    assert np.abs(bad["Y"] - good["Y"]).max() > 1e-3
