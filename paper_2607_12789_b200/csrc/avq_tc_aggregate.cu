@@ -1,5 +1,9 @@
 // Value aggregation for the bf16 path (Eq. "aggregates"; the scatter steps of Algorithm 1).
 //
+// (After a bounded wait has expired in the assign kernel its indices are meaningless but in range, so these
+// kernels run on regardless - they only flag indices that are out of range - and the attention kernel,
+// which reads the status word, leaves without writing.)
+//
 // leaf_scatter_kernel  one warp per 8 keys: each key's V row is added to the sum of its leaf
 //                      codeword (parent, child) with vector reductions to global memory, and
 //                      the leaf's count is bumped.  Only the leaf level is scattered; a key whose
@@ -52,8 +56,6 @@ leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restri
   }
   tc::pdl_wait();                                    // the indices come from the kernel before
   if (j0 >= Nk) return;
-  // an earlier kernel of this call gave up on a wait: its indices are not valid, do not scatter them
-  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word) != 0) return;
   // leaf_l: a * C + c for a key that moved to child c, kStayBit | a for a key that stays, -1 = nothing to add
   constexpr int kStayBit = 1 << 30;
   int leaf_l = -1;
@@ -120,8 +122,6 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
   __syncthreads();
   tc::pdl_wait();                                      // the indices come from the kernel before
   if (n <= 0) return;
-  // an earlier kernel of this call gave up on a wait: its indices are not valid, do not scatter them
-  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word) != 0) return;
   const size_t kb = (size_t)bh * Nk + j0;
 
   // ---- leaf of every key and its rank among the chunk's keys of that leaf
@@ -230,60 +230,57 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
   flush();
 }
 
-// One CTA: 8 consecutive parents of one (batch, head); thread k owns head-dimension index k.
-// 32 loads per thread are issued before their first use.
+// One CTA: kPer consecutive parents of one (batch, head) (8 with four children each, 4 with eight: 32 leaf
+// rows); thread k owns head-dimension index k.  Every load is issued before the first use.
 template <int D, int C>
 __global__ void __launch_bounds__(D)
 finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, float* __restrict__ Vp,
                 float* __restrict__ np_, __nv_bfloat16* __restrict__ Vpb, __nv_bfloat16* __restrict__ Vcb,
-                __nv_bfloat16* __restrict__ Vsb, float* __restrict__ rho, int M, const int32_t* status_word) {
+                __nv_bfloat16* __restrict__ Vsb, float* __restrict__ rho, int M) {
+  constexpr int kPer = (C == 4) ? 8 : 4;
   tc::pdl_launch_dependents();
   tc::pdl_wait();                                    // the leaf sums come from the kernel before
-  if (status_word && *reinterpret_cast<const volatile int32_t*>(status_word) != 0) return;
-  const int bh = blockIdx.y, m0 = blockIdx.x * 8, k = threadIdx.x;
-  constexpr int kPer = (C == 4) ? 8 : 4;             // parents whose loads are in flight together (32 floats)
+  const int bh = blockIdx.y, m0 = blockIdx.x * kPer, k = threadIdx.x;
+  float x[kPer][C], cn[kPer][C], stay[kPer], nstay[kPer];
 #pragma unroll
-  for (int g = 0; g < 8 / kPer; ++g) {
-    // every load of the group is issued before the first use
-    float x[kPer][C], cn[kPer][C], stay[kPer], nstay[kPer];
+  for (int mm = 0; mm < kPer; ++mm) {
+    const size_t row = (size_t)bh * M + m0 + mm;
 #pragma unroll
-    for (int mm = 0; mm < kPer; ++mm) {
-      const size_t row = (size_t)bh * M + m0 + g * kPer + mm;
-#pragma unroll
-      for (int c = 0; c < C; ++c) {
-        x[mm][c] = Vc[(row * C + c) * D + k];
-        cn[mm][c] = nc[row * C + c];
-      }
-      stay[mm] = Vp[row * D + k];                      // accumulated by the scatter (zero unless keys stay)
-      nstay[mm] = np_[row];                            // keys that stay (the total is written after the barrier below)
+    for (int c = 0; c < C; ++c) {
+      x[mm][c] = Vc[(row * C + c) * D + k];
+      cn[mm][c] = nc[row * C + c];
     }
+    // The stay accumulators are read AND rewritten by this kernel; volatile loads pin the reads behind the
+    // dependency wait above (a plain load of np_ was seen to be scheduled ahead of it, reading counts the
+    // scatter had not finished).
+    stay[mm] = *reinterpret_cast<const volatile float*>(Vp + row * D + k);   // zero unless keys stay
+    nstay[mm] = *reinterpret_cast<const volatile float*>(np_ + row);         // keys that stay
+  }
+  float ntot[kPer];
 #pragma unroll
-    for (int mm = 0; mm < kPer; ++mm) {
-      const size_t row = (size_t)bh * M + m0 + g * kPer + mm;
-      float s = stay[mm], n = nstay[mm];
+  for (int mm = 0; mm < kPer; ++mm) {
+    const size_t row = (size_t)bh * M + m0 + mm;
+    float s = stay[mm], n = nstay[mm];
 #pragma unroll
-      for (int c = 0; c < C; ++c) {
-        s += x[mm][c];
-        n += cn[mm][c];
-        // the attention kernels take per-codeword MEANS: the count rides in their softmax weights
-        if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(cn[mm][c] > 0.f ? x[mm][c] * __frcp_rn(cn[mm][c]) : 0.f);
-      }
-      Vp[row * D + k] = s;
-      const float rn = n > 0.f ? __frcp_rn(n) : 0.f;
-      if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(s * rn);
-      // what a refined parent keeps under the PARENT_STAYS rule, per key of the parent: its weight in the
-      // attention kernel is A n_p, so the row is Vbar_stay / n_p and the count n_stay / n_p
-      if (Vsb) Vsb[row * D + k] = __float2bfloat16_rn(stay[mm] * rn);
-      if (rho && k == 0) rho[row] = nstay[mm] * rn;
+    for (int c = 0; c < C; ++c) {
+      s += x[mm][c];
+      n += cn[mm][c];
+      // the attention kernel takes per-codeword MEANS: the count rides in its softmax weights
+      if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(cn[mm][c] > 0.f ? x[mm][c] * __frcp_rn(cn[mm][c]) : 0.f);
     }
+    ntot[mm] = n;
+    Vp[row * D + k] = s;
+    const float rn = n > 0.f ? __frcp_rn(n) : 0.f;
+    if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(s * rn);
+    // what a refined parent keeps under the PARENT_STAYS rule, per key of the parent: its weight in the
+    // attention kernel is A n_p, so the row is Vbar_stay / n_p and the count n_stay / n_p
+    if (Vsb) Vsb[row * D + k] = __float2bfloat16_rn(stay[mm] * rn);
+    if (rho && k == 0) rho[row] = nstay[mm] * rn;
   }
   __syncthreads();                                     // every thread has read the stay counts
-  if (k < 8) {
-    const int m = m0 + k;
-    float s = np_[(size_t)bh * M + m];                 // keys that stay with the parent
+  if (k == 0) {
 #pragma unroll
-    for (int c = 0; c < C; ++c) s += nc[((size_t)bh * M + m) * C + c];
-    np_[(size_t)bh * M + m] = s;
+    for (int mm = 0; mm < kPer; ++mm) np_[(size_t)bh * M + m0 + mm] = ntot[mm];
   }
 }
 
@@ -343,11 +340,10 @@ avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const i
                        status_word) != cudaSuccess)
       return AVQ_ERR_CUDA;
   }
-  dim3 g2(p.M / 8, BH);
+  dim3 g2(p.M / (C == 4 ? 8 : 4), BH);
   return cuda_ok(tc::launch_pdl(finalize_kernel<D, C>, g2, dim3(D), 0, st, true, static_cast<const float*>(Vc),
                                 static_cast<const float*>(nc), Vp, np_, static_cast<__nv_bfloat16*>(Vpb),
-                                static_cast<__nv_bfloat16*>(Vcb), static_cast<__nv_bfloat16*>(Vsb), rho, p.M,
-                                static_cast<const int32_t*>(status_word)));
+                                static_cast<__nv_bfloat16*>(Vcb), static_cast<__nv_bfloat16*>(Vsb), rho, p.M));
 }
 
 }  // namespace

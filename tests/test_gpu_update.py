@@ -25,8 +25,10 @@ def _state(wl, seed):
                                       (synth.C0.with_(B=2, H=2, seed=22, keys_around_parents=True, sigma_k=0.4),
                                        binding.FLAG_PARENT_STAYS),
                                       (synth.C1.with_(B=2, H=3, N=2000, seed=23), 0),
-                                      (synth.C3.with_(B=1, H=2, N=3000, seed=24), 0)],
-                         ids=["f32", "f32_parent_stays", "bf16_d64", "bf16_d128_M256"])
+                                      (synth.C3.with_(B=1, H=2, N=3000, seed=24), 0),
+                                      (synth.C1.with_(B=2, H=2, N=1500, seed=25, keys_around_parents=True,
+                                                      sigma_k=0.45), binding.FLAG_PARENT_STAYS)],
+                         ids=["f32", "f32_parent_stays", "bf16_d64", "bf16_d128_M256", "bf16_parent_stays"])
 def test_update_matches_the_oracle(wl, flags):
     x = synth.generate(wl)
     Sp, Np, Sc, Nc = _state(wl, wl.seed)
