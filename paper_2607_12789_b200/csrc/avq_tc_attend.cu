@@ -5,10 +5,12 @@
 // Flow of a tile:
 //   parents   S = Q . Cp^T                 tcgen05.mma, fp32 accumulator in TMEM columns [0, M)
 //             read once into registers: row maximum over non-empty parents, exp2, exact
-//             denominator z                                         (Eq. "vqflashattention")
+//             denominator z                                         (Eq. "vqflashattention");
+//             in the same loop the bf16 weights A_ij n_j -> shared memory (over the dead codebook)
 //             importance w_j = n_j sum_i A_ij / z_i from the fp32 weights  (Eq. "importance")
 //             top-P by rank, ties to the lower index                ("Child spawning")
-//             bf16 weights A_ij n_j -> shared memory; a refined parent's row of the value tile is cleared
+//             a refined parent's row of the value tile becomes its stay row (zeros by default) and its
+//             rounded weights leave the denominator
 //             O = (A n) . mean_p           tcgen05.mma into TMEM columns [CT, CT + d)
 //   children  of the selected parents, in chunks of <= CHW columns: gathered codeword rows,
 //             S_c = Q . Cc_sel^T, running maximum (non-empty children only), O rescaled in TMEM if a
@@ -16,8 +18,9 @@
 //   Y = O / z, z accumulated from the same bf16-rounded weights as the numerator.
 // Empty codewords are excluded from every maximum and contribute nothing (their count and value sum
 // are zero; their weight is clamped so that it stays finite) - appendix on numerical stability.
-// The gathers of the first child chunk are issued early so that their latency hides behind the weight
-// conversion and the parents' second MMA.
+// The gathers of the first child chunk are issued as soon as the selection is known.  With one CTA per SM
+// (CT = 256) the next tile's codebook is loaded into the halves of the weight and value tiles that the child
+// phase leaves free, and the next tile's S is issued before this tile's epilogue.
 #include "avq_tc_common.cuh"
 
 namespace avq {
@@ -89,23 +92,21 @@ __device__ __forceinline__ void row_sync(int q) {
 
 // Multiplies 16 fp32 weights by their codewords' key counts, rounds the products to bf16, stores them at
 // (row r, columns col0..col0+15) of the K-major swizzled A tile, and returns the sum of the rounded
-// products times a 0/1 mask (`keep16`: 0 for a refined parent, whose value row has been cleared).
+// products (the denominator is built from exactly what the value MMA multiplies).
 __device__ __forceinline__ float store_weights16(unsigned char* A, int r, int col0, const float* cnt16,
-                                                 const float* keep16, const float (&a)[16]) {
+                                                 const float (&a)[16]) {
   const float4* n4 = reinterpret_cast<const float4*>(cnt16);
-  const float4* k4 = reinterpret_cast<const float4*>(keep16);
   uint32_t pk[8];
-  float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;         // independent partial sums: no 16-deep FMA chain
+  float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;         // independent partial sums: no 16-deep add chain
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
     const float4 n = n4[u];
-    const float4 k = k4[u];
     const uint32_t p0 = pack_bf16(a[4 * u] * n.x, a[4 * u + 1] * n.y);
     const uint32_t p1 = pack_bf16(a[4 * u + 2] * n.z, a[4 * u + 3] * n.w);
-    z0 = fmaf(__uint_as_float(p0 << 16), k.x, z0);
-    z1 = fmaf(__uint_as_float(p0 & 0xFFFF0000u), k.y, z1);
-    z2 = fmaf(__uint_as_float(p1 << 16), k.z, z2);
-    z3 = fmaf(__uint_as_float(p1 & 0xFFFF0000u), k.w, z3);
+    z0 += __uint_as_float(p0 << 16);
+    z1 += __uint_as_float(p0 & 0xFFFF0000u);
+    z2 += __uint_as_float(p1 << 16);
+    z3 += __uint_as_float(p1 & 0xFFFF0000u);
     pk[2 * u] = p0;
     pk[2 * u + 1] = p1;
   }
@@ -144,17 +145,17 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   unsigned char* CC = Vs + subA * D * 128;               // kSubD x [CHW x 128 B] gathered child codes
   float* cnt = reinterpret_cast<float*>(CC + CHW * D * 2);   // [CT] key counts of the parents
   float* bias = cnt + CT;                                // [CT] 0 for non-empty parents, -inf for empty
-  float* cntk = bias + CT;                               // [CT] 1 for a parent that keeps its own term, 0 once refined
+  float* cntk = bias + CT;                               // [CT] share of its own term a parent keeps: 1, or once refined 0 / its stay share
   float* cntc = cntk + CT;                               // [CHW] key counts of the child chunk
   float* biasc = cntc + CHW;                             // [CHW]
-  float* keepc = biasc + CHW;                            // [CHW] all ones (children are never removed)
-  float* w = keepc + CHW;                                // [256] importance
-  float* wpart = w + 256;                                // [4][CT]
+  float* w = biasc + CHW;                                // [CT] importance
+  float* wpart = w + CT;                                 // [4][CT]
   float* xm = wpart + 4 * CT;                            // [NQ][128] exchange between the threads of a row
   float* xz = xm + NQ * kRows;                           // [NQ][128]
   float* xz2 = xz + NQ * kRows;                          // [NQ][128]
-  int* sel_list = reinterpret_cast<int*>(xz2 + NQ * kRows);   // [256]
-  uint32_t* wmask = reinterpret_cast<uint32_t*>(sel_list + 256);   // [16]
+  float* ncs = xz2 + NQ * kRows;                         // [M * C] key counts of every child of this (b, h)
+  int* sel_list = reinterpret_cast<int*>(ncs + p.M * p.C);    // [CT]
+  uint32_t* wmask = reinterpret_cast<uint32_t*>(sel_list + CT);    // [16]
   uint64_t* bars = reinterpret_cast<uint64_t*>(wmask + 18);        // [5]  (wmask[16] is a scratch word)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -175,6 +176,18 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // buffer, which are adjacent and together as large (the next tile's value rows then load a little later).
   constexpr bool kChain = true;
   constexpr bool kStageInCC = CT >= 128;
+  // CT = 256 (one CTA per SM) with children to refine: the child phase uses only the lower half of the weight
+  // tile and of the value tile (a chunk is at most 128 columns / rows), so the NEXT tile's codebook is loaded
+  // into the upper halves as soon as the parents' value MMA has finished, and the next tile's S = Q . Cp^T is
+  // issued right after the last child logits have been read: it runs under the epilogue instead of
+  // opening the next tile with a load -> MMA chain everyone waits for.
+  constexpr bool kEarlySCap = (CT == 256);
+  const bool early_s = kEarlySCap && p.P > 0;
+  constexpr int kVsBytes = subA * D * 128;
+  auto cp_sub = [&](int s) -> unsigned char* {           // where sub-tile s (64 columns) of the codebook lives
+    if (!early_s) return CA + s * (p.M * 128);
+    return s == 0 ? CA + ca_bytes / 2 : Vs + kVsBytes / 2;
+  };
   static_assert(kStageInCC || (CT * D * 2 + CHW * D * 2 == kSubD * kRows * 128), "staging area");
   auto issue_q = [&](int t) {                            // thread 0 only
     const int tb = t / p.nblk, ti0 = (t - tb * p.nblk) * kRows;
@@ -186,13 +199,28 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int th = (t / p.nblk) % p.H;
     mbar_expect_tx(bar_cp, (uint32_t)(kSubD * M * 128));
 #pragma unroll
-    for (int s = 0; s < kSubD; ++s) tma_load_2d(CA + s * M * 128, &tmCp, s * 64, th * M, bar_cp);
+    for (int s = 0; s < kSubD; ++s) tma_load_2d(cp_sub(s), &tmCp, s * 64, th * M, bar_cp);
   };
   auto issue_vp = [&](int t) {
     const int tb = t / p.nblk;
     mbar_expect_tx(bar_ld1, (uint32_t)(kSubD * M * 128));
 #pragma unroll
     for (int s = 0; s < kSubD; ++s) tma_load_2d(Vs + s * M * 128, &tmVpb, s * 64, tb * M, bar_ld1);
+  };
+
+  auto issue_s = [&](uint32_t tmem_d, uint32_t parity) {  // one thread: S = Q . Cp^T once both tiles have landed
+    const bool q_ok = mbar_wait(bar_q, parity, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+    const bool c_ok = mbar_wait(bar_cp, parity, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
+    if (q_ok && c_ok) {
+      tc_fence_after();
+      const uint32_t idesc = umma_idesc_bf16(kRows, M);
+      const uint32_t qa = smem_u32(Qs);
+#pragma unroll
+      for (int k = 0; k < D / 16; ++k)
+        umma_bf16(tmem_d, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
+                  umma_desc_sw128(smem_u32(cp_sub(k / 4)) + (k % 4) * 32), idesc, k > 0);
+    }
+    umma_commit(bar_s);
   };
 
   __shared__ int early_exit;
@@ -240,18 +268,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int next_tile = tile + gridDim.x;
   const bool has_next = kChain && next_tile < p.total_tiles;
   if (tid == 0) {
-    const bool q_ok = mbar_wait(bar_q, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
-    const bool c_ok = mbar_wait(bar_cp, ph_in, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
-    if (q_ok && c_ok) {
-      tc_fence_after();
-      const uint32_t idesc = umma_idesc_bf16(kRows, M);
-      const uint32_t qa = smem_u32(Qs), ca = smem_u32(CA);
-#pragma unroll
-      for (int k = 0; k < D / 16; ++k)
-        umma_bf16(tmem_base, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
-                  umma_desc_sw128(ca + (k / 4) * M * 128 + (k % 4) * 32), idesc, k > 0);
-    }
-    umma_commit(bar_s);
+    if (!early_s || first) issue_s(tmem_base, ph_in);   // otherwise issued during the tile before
     if (!kStageInCC && !first) {
       // the value tile was the staging area of the tile before: reload it once that store has read it
       tma_store_wait_read();
@@ -266,7 +283,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (tid == 0) {
       // a wait that expired in an earlier CTA or kernel of this call: do not start more work
       early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
-      issue_vp(tile);
+      if (!early_s) issue_vp(tile);                    // early_s: the value tile still holds half of the codebook
     }
   }
   for (int j = tid; j < CT; j += kThreads) {
@@ -275,11 +292,16 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     bias[j] = n > 0.f ? 0.f : -INFINITY;
     cntk[j] = 1.f;
   }
+  // every child's key count: the gathers below pick theirs from shared memory instead of waiting for a
+  // dependent global load once the selection is known
+  if (PC > 0)
+    for (int j = tid; j < ((M * C) >> 2); j += kThreads)
+      reinterpret_cast<float4*>(ncs)[j] = __ldg(reinterpret_cast<const float4*>(p.nc + (size_t)bh * M * C) + j);
   __syncthreads();
   if (first && early_exit) {
     // let the MMA and the load already in flight finish, then leave cleanly
     mbar_wait(bar_s, 0, abort_flag, nullptr, 0);
-    mbar_wait(bar_ld1, 0, abort_flag, nullptr, 0);
+    if (!early_s) mbar_wait(bar_ld1, 0, abort_flag, nullptr, 0);
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
@@ -292,6 +314,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   ph_s ^= 1;
   tc_fence_after();
   if (tid == 0 && has_next && PC == 0) issue_q(next_tile);   // no child logits will read this Q tile
+  if (tid == 0 && early_s) issue_vp(tile);              // S is done and so is the last value MMA of the tile before
   // This thread's QW (<= 64) parent logits are read from TMEM once and stay in registers through the
   // maximum, the exponentials, the importance sums and the conversion to bf16.
   float a[QW];
@@ -329,7 +352,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
   // ---- fp32 weights; exact denominator of the parent pass.  Empty parents carry a logit of -inf, hence
   // a weight of exactly zero; every other logit is at most the maximum (up to one rounding).
-  float zfull = 0.f;
+  float zfull = 0.f, zall = 0.f;                          // zall: sum of this thread's bf16-rounded weights x counts
   {
     float zf0 = 0.f, zf1 = 0.f, zf2 = 0.f, zf3 = 0.f;
     const float negm = -m_run;
@@ -349,6 +372,13 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           zf2 = fmaf(a[c0 + 4 * u + 2], n.z, zf2);
           zf3 = fmaf(a[c0 + 4 * u + 3], n.w, zf3);
         }
+        // The bf16 weights go to shared memory (over the dead codebook) right here: the exponentials keep the
+        // XU pipe busy and the conversion (ALU pipe, stores) fills the issue slots they leave empty.  The
+        // selection is not known yet; what it removes is taken out of the denominator afterwards.
+        float am[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) am[e] = a[c0 + e];
+        zall += store_weights16(CA, r, colbase + c0, cnt + colbase + c0, am);
       }
     }
     zfull = (zf0 + zf1) + (zf2 + zf3);
@@ -472,7 +502,6 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // ---- first child chunk: start the asynchronous gather of its codeword rows now; it lands while the
   // weight conversion below runs
   const __nv_bfloat16* Cch = p.Cc + (size_t)h * M * C * D;
-  const float* ncb = p.nc + (size_t)bh * M * C;
   int ncols = min(PC, CHW);
   int np16 = (ncols + 15) & ~15;
   // Rows of a chunk, gathered into a K-major / row-per-codeword tile of np16 rows (kSubD sub-tiles of 64
@@ -480,31 +509,39 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // A thread keeps its 16-byte chunk column and walks down the rows (kThreads is a multiple of the chunks
   // per row).
   auto gather_rows = [&](unsigned char* tile, const __nv_bfloat16* src, int e_first) {
-    constexpr int kRowsPerPass = kThreads >> kLogChunks;
-    const int ch = tid & ((1 << kLogChunks) - 1);
-    const uint32_t dst_col = (uint32_t)((ch >> 3) * (np16 * 128));
+    constexpr int kRowsPerPass = kThreads >> kLogChunks;   // a multiple of 8: a thread's swizzle phase is fixed
+    constexpr int kPasses = (CHW + kRowsPerPass - 1) / kRowsPerPass;
+    const int ch = tid & ((1 << kLogChunks) - 1), row0 = tid >> kLogChunks;
+    const uint32_t dst0 = smem_u32(tile) + (uint32_t)((ch >> 3) * (np16 * 128)) + sw128_offset(row0, (ch & 7) * 8);
     const __nv_bfloat16* src_col = src + ch * 8;
-    for (int row = tid >> kLogChunks; row < np16; row += kRowsPerPass) {
-      unsigned char* dst = tile + dst_col + sw128_offset(row, (ch & 7) * 8);
+    int sel[kPasses];
+#pragma unroll
+    for (int it = 0; it < kPasses; ++it) {                 // the list look-ups first, all in flight together
+      const int e = e_first + row0 + it * kRowsPerPass;
+      sel[it] = (row0 + it * kRowsPerPass < ncols) ? sel_list[e >> logC] : 0;
+    }
+#pragma unroll
+    for (int it = 0; it < kPasses; ++it) {
+      const int row = row0 + it * kRowsPerPass;
+      const uint32_t dst = dst0 + (uint32_t)(it * kRowsPerPass * 128);
       if (row < ncols) {
         const int e = e_first + row;
-        cp_async16(dst, src_col + (((size_t)sel_list[e >> logC] << logC) + (e & (C - 1))) * D);
-      } else {
-        *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+        const uint32_t off = (uint32_t)(((sel[it] << logC) + (e & (C - 1))) << kLogD);   // elements: < 2^31
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src_col + off) : "memory");
+      } else if (row < np16) {
+        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
       }
     }
   };
   auto gather_codes = [&](int e_first) {
-    // the child counts are fetched first so that their latency hides behind the copies
     float n_child = 0.f;
     if (tid < ncols) {                                   // CHW <= 128 <= kThreads
       const int e = e_first + tid;
-      n_child = __ldg(ncb + ((size_t)sel_list[e >> logC] << logC) + (e & (C - 1)));
+      n_child = ncs[(sel_list[e >> logC] << logC) + (e & (C - 1))];
     }
     gather_rows(CC, Cch, e_first);
     if (tid < CHW) {
       cntc[tid] = n_child;
-      keepc[tid] = 1.f;
       biasc[tid] = n_child > 0.f ? 0.f : -INFINITY;
     }
   };
@@ -524,17 +561,17 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     *reinterpret_cast<uint4*>(Vs + (ch >> 3) * (M * 128) + sw128_offset(row, (ch & 7) * 8)) = stay;
   }
   {
-    float zloc = 0.f;
-#pragma unroll
-    for (int c0 = 0; c0 < QW; c0 += 16) {
-      if (c0 < my_cols) {
-        float am[16];
-#pragma unroll
-        for (int e = 0; e < 16; ++e) am[e] = a[c0 + e];
-        zloc += store_weights16(CA, r, colbase + c0, cnt + colbase + c0, cntk + colbase + c0, am);
-      }
+    // denominator of the parent pass from the rounded weights, less what the refined parents no longer carry
+    // (all of it under the default rule, the share of the keys that moved to children under PARENT_STAYS);
+    // the row's NQ threads split the P look-ups
+    float fix = 0.f;
+    for (int u = cq; u < min(P, M); u += NQ) {
+      const int j = sel_list[u];
+      const uint16_t hv =
+          *reinterpret_cast<const uint16_t*>(CA + (j >> 6) * (kRows * 128) + sw128_offset(r, j & 63));
+      fix = fmaf(__uint_as_float((uint32_t)hv << 16), 1.f - cntk[j], fix);
     }
-    xz2[cq * kRows + r] = zloc;
+    xz2[cq * kRows + r] = zall - fix;
   }
   cp_async_wait_all();
   fence_proxy_async();
@@ -575,6 +612,8 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     mbar_wait(bar_pv, ph_pv, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
     ph_pv ^= 1;
     tc_fence_after();
+    // the parents' value MMA is done: the upper halves of the weight tile and of the value tile are free
+    if (tid == 0 && early_s && has_next && e0 == 0) issue_cp(next_tile);
     // value rows of this chunk (the same gather as for its codeword rows).  Asynchronous copies: they land
     // while the chunk's logits are turned into weights.  Padding rows are zero: they meet finite weights.
     gather_rows(Vs, Vch, e0);
@@ -632,7 +671,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         tmem_ld16(t_sc + c0, a);
 #pragma unroll
         for (int e = 0; e < 16; ++e) a[e] = ex2(fminf(fmaf(a[e], sc, negm), kLazyLog2));   // clamp: empty children
-        zloc += store_weights16(CA, r, cq * QWC + c0, cntc + cq * QWC + c0, keepc + cq * QWC + c0, a);
+        zloc += store_weights16(CA, r, cq * QWC + c0, cntc + cq * QWC + c0, a);
       }
       xz2[cq * kRows + r] = zloc;
     }
@@ -671,6 +710,9 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     umma_desc_sw128(ca + (k / 4) * np16 * 128 + (k % 4) * 32), idesc, k > 0);
         umma_commit(bar_s);
       }
+    } else if (tid == kScLane && early_s && has_next) {
+      // every thread has read the last child logits (barrier above): the next tile's parent logits
+      issue_s(tmem_base, ph_in ^ 1);
     }
   }
 
@@ -680,7 +722,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tc_fence_after();
   // the last value MMA has released the weight tile and the value tile: the next tile's codebook and
   // parent value rows load while this tile's output is written
-  if (tid == 0 && has_next) {
+  if (tid == 0 && has_next && !early_s) {
     issue_cp(next_tile);
     if (kStageInCC) issue_vp(next_tile);
   }
@@ -716,13 +758,13 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
 }
 
-size_t attend_smem(int D, int CT, int CHW, int NQ) {
+size_t attend_smem(int D, int CT, int CHW, int NQ, int MC) {
   const int subA = CT / 64;
   const size_t ca = (size_t)max(CT * D * 2, subA * kRows * 128);
   size_t b = (size_t)(D / 64) * kRows * 128 + ca + (size_t)subA * D * 128 + (size_t)CHW * D * 2;
-  b += sizeof(float) * (3 * (size_t)CT + 3 * (size_t)CHW + 256 + 4 * (size_t)CT + 3 * (size_t)NQ * kRows);
-  b += sizeof(int) * 256 + sizeof(uint32_t) * 18 + sizeof(uint64_t) * 5 + 2 * sizeof(uint32_t);
-  return b + 64;
+  b += sizeof(float) * (3 * (size_t)CT + 2 * (size_t)CHW + (size_t)CT + 4 * (size_t)CT + 3 * (size_t)NQ * kRows);
+  b += sizeof(int) * (size_t)CT + sizeof(uint32_t) * 18 + sizeof(uint64_t) * 5 + 2 * sizeof(uint32_t);
+  return b + 64 + sizeof(float) * (size_t)MC;
 }
 
 template <int D, int NQ, int CT>
@@ -804,7 +846,7 @@ avq_status launch(const avq_problem& p, const void* Q, const void* Cp, const voi
   a.tmem_cols = cols;
   a.scale_log2e = p.scale * 1.4426950408889634f;
   const int NQ = (D == 64) ? (CT == 64 ? 1 : (CT == 128 ? 2 : 4)) : (CT == 64 ? 2 : 4);
-  const size_t smem = attend_smem(D, CT, CHW, NQ);
+  const size_t smem = attend_smem(D, CT, CHW, NQ, p.M * p.C);
   // Threads per query row follow from how many CTAs can share an SM (TMEM columns, shared memory):
   // four small CTAs of 128 threads, two of 256, or one of 512.
   const unsigned bh = (unsigned)BH;
