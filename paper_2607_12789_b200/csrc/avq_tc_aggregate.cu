@@ -60,8 +60,8 @@ leaf_scatter_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restri
   constexpr int kStayBit = 1 << 30;
   int leaf_l = -1;
   if (lane < kKeysPerWarp && j0 + lane < Nk) {
-    const int a = __ldg(pidx + kb + j0 + lane);
-    const int c = __ldg(cidx + kb + j0 + lane);
+    const int a = tc::ld_after_wait(pidx + kb + j0 + lane);   // ordered behind the dependency wait
+    const int c = tc::ld_after_wait(cidx + kb + j0 + lane);
     if (a < 0 || a >= M || c < -1 || c >= C) {       // caller-supplied index out of range: skip the key, flag it
       if (status_word) atomicCAS(status_word, 0, DEV_BAD_INDEX);
     } else {
@@ -131,7 +131,7 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
     const int j = tid + t * kSortThreads;
     lr[t] = 0xFFFFFFFFu;
     if (j < n) {
-      const int a = __ldg(pidx + kb + j), c = __ldg(cidx + kb + j);
+      const int a = tc::ld_after_wait(pidx + kb + j), c = tc::ld_after_wait(cidx + kb + j);   // behind the wait
       if (a < 0 || a >= M || c < -1 || c >= C) {       // caller-supplied index out of range: skip the key, flag it
         if (status_word) atomicCAS(status_word, 0, DEV_BAD_INDEX);
       } else {
@@ -247,14 +247,14 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
     const size_t row = (size_t)bh * M + m0 + mm;
 #pragma unroll
     for (int c = 0; c < C; ++c) {
-      x[mm][c] = Vc[(row * C + c) * D + k];
-      cn[mm][c] = nc[row * C + c];
+      x[mm][c] = tc::ld_after_wait(Vc + (row * C + c) * D + k);
+      cn[mm][c] = tc::ld_after_wait(nc + row * C + c);
     }
-    // The stay accumulators are read AND rewritten by this kernel; volatile loads pin the reads behind the
-    // dependency wait above (a plain load of np_ was seen to be scheduled ahead of it, reading counts the
-    // scatter had not finished).
-    stay[mm] = *reinterpret_cast<const volatile float*>(Vp + row * D + k);   // zero unless keys stay
-    nstay[mm] = *reinterpret_cast<const volatile float*>(np_ + row);         // keys that stay
+    // Everything read here is written by the kernel before this one: the loads are statements the compiler
+    // cannot move ahead of the dependency wait above (an ordinary load of np_ was seen to be scheduled ahead
+    // of it, reading counts the scatter had not finished).
+    stay[mm] = tc::ld_after_wait(Vp + row * D + k);   // zero unless keys stay
+    nstay[mm] = tc::ld_after_wait(np_ + row);         // keys that stay
   }
   float ntot[kPer];
 #pragma unroll

@@ -18,9 +18,7 @@
 //   Y = O / z, z accumulated from the same bf16-rounded weights as the numerator.
 // Empty codewords are excluded from every maximum and contribute nothing (their count and value sum
 // are zero; their weight is clamped so that it stays finite) - appendix on numerical stability.
-// The gathers of the first child chunk are issued as soon as the selection is known.  With one CTA per SM
-// (CT = 256) the next tile's codebook is loaded into the halves of the weight and value tiles that the child
-// phase leaves free, and the next tile's S is issued before this tile's epilogue.
+// The gathers of the first child chunk are issued as soon as the selection is known.
 #include "avq_tc_common.cuh"
 
 namespace avq {
@@ -176,19 +174,6 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // buffer, which are adjacent and together as large (the next tile's value rows then load a little later).
   constexpr bool kChain = true;
   constexpr bool kStageInCC = CT >= 128;
-  // CT = 256 (one CTA per SM) with children to refine: the child phase uses only the lower half of the weight
-  // tile and of the value tile (a chunk is at most 128 columns / rows), so the NEXT tile's codebook is loaded
-  // into the upper halves as soon as the parents' value MMA has finished, and the next tile's S = Q . Cp^T is
-  // issued right after the last child logits have been read: it runs under the epilogue instead of
-  // opening the next tile with a load -> MMA chain everyone waits for.
-  constexpr bool kEarlySCap = (CT == 256);
-  const bool early_s = kEarlySCap && p.P > 0;
-  constexpr int kVsBytes = subA * D * 128;
-  auto cp_sub = [&](int s) -> unsigned char* {           // where sub-tile s (64 columns) of the codebook lives
-    if (!early_s) return CA + s * (p.M * 128);
-    return s == 0 ? CA + ca_bytes / 2 : Vs + kVsBytes / 2;
-  };
-  static_assert(kStageInCC || (CT * D * 2 + CHW * D * 2 == kSubD * kRows * 128), "staging area");
   auto issue_q = [&](int t) {                            // thread 0 only
     const int tb = t / p.nblk, ti0 = (t - tb * p.nblk) * kRows;
     mbar_expect_tx(bar_q, (uint32_t)(kSubD * kRows * 128));
@@ -199,7 +184,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int th = (t / p.nblk) % p.H;
     mbar_expect_tx(bar_cp, (uint32_t)(kSubD * M * 128));
 #pragma unroll
-    for (int s = 0; s < kSubD; ++s) tma_load_2d(cp_sub(s), &tmCp, s * 64, th * M, bar_cp);
+    for (int s = 0; s < kSubD; ++s) tma_load_2d(CA + s * M * 128, &tmCp, s * 64, th * M, bar_cp);
   };
   auto issue_vp = [&](int t) {
     const int tb = t / p.nblk;
@@ -214,11 +199,11 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (q_ok && c_ok) {
       tc_fence_after();
       const uint32_t idesc = umma_idesc_bf16(kRows, M);
-      const uint32_t qa = smem_u32(Qs);
+      const uint32_t qa = smem_u32(Qs), ca = smem_u32(CA);
 #pragma unroll
       for (int k = 0; k < D / 16; ++k)
         umma_bf16(tmem_d, umma_desc_sw128(qa + (k / 4) * kRows * 128 + (k % 4) * 32),
-                  umma_desc_sw128(smem_u32(cp_sub(k / 4)) + (k % 4) * 32), idesc, k > 0);
+                  umma_desc_sw128(ca + (k / 4) * M * 128 + (k % 4) * 32), idesc, k > 0);
     }
     umma_commit(bar_s);
   };
@@ -267,8 +252,21 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int rows_valid = min(kRows, p.Nq - i0);
   const int next_tile = tile + gridDim.x;
   const bool has_next = kChain && next_tile < p.total_tiles;
+  // Key counts of this (b, h): one parent count and one 16-byte group of child counts per thread.  Their loads
+  // are started before thread 0 turns to the MMA issue so that its warp is not a load latency behind the
+  // others at the next barrier (first tile: only after the dependency wait below - the kernel before this
+  // one writes them, so they are loaded with statements the compiler cannot move ahead of that wait).
+  static_assert(CT <= kThreads && 2 * CT <= 4 * kThreads, "one count load per thread");
+  float n_reg = 0.f;
+  float4 nc_reg = make_float4(0.f, 0.f, 0.f, 0.f);
+  auto load_counts = [&]() {
+    if (tid < M) n_reg = ld_after_wait(p.np_ + (size_t)bh * M + tid);
+    if (PC > 0 && tid < ((M * C) >> 2))
+      nc_reg = ld_after_wait(reinterpret_cast<const float4*>(p.nc + (size_t)bh * M * C) + tid);
+  };
+  if (!first) load_counts();
   if (tid == 0) {
-    if (!early_s || first) issue_s(tmem_base, ph_in);   // otherwise issued during the tile before
+    issue_s(tmem_base, ph_in);
     if (!kStageInCC && !first) {
       // the value tile was the staging area of the tile before: reload it once that store has read it
       tma_store_wait_read();
@@ -283,25 +281,23 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (tid == 0) {
       // a wait that expired in an earlier CTA or kernel of this call: do not start more work
       early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
-      if (!early_s) issue_vp(tile);                    // early_s: the value tile still holds half of the codebook
+      issue_vp(tile);
     }
+    load_counts();
   }
-  for (int j = tid; j < CT; j += kThreads) {
-    const float n = j < M ? p.np_[(size_t)bh * M + j] : 0.f;
-    cnt[j] = n;
-    bias[j] = n > 0.f ? 0.f : -INFINITY;
-    cntk[j] = 1.f;
+  if (tid < CT) {
+    cnt[tid] = n_reg;
+    bias[tid] = n_reg > 0.f ? 0.f : -INFINITY;
+    cntk[tid] = 1.f;
   }
   // every child's key count: the gathers below pick theirs from shared memory instead of waiting for a
   // dependent global load once the selection is known
-  if (PC > 0)
-    for (int j = tid; j < ((M * C) >> 2); j += kThreads)
-      reinterpret_cast<float4*>(ncs)[j] = __ldg(reinterpret_cast<const float4*>(p.nc + (size_t)bh * M * C) + j);
+  if (PC > 0 && tid < ((M * C) >> 2)) reinterpret_cast<float4*>(ncs)[tid] = nc_reg;
   __syncthreads();
   if (first && early_exit) {
     // let the MMA and the load already in flight finish, then leave cleanly
     mbar_wait(bar_s, 0, abort_flag, nullptr, 0);
-    if (!early_s) mbar_wait(bar_ld1, 0, abort_flag, nullptr, 0);
+    mbar_wait(bar_ld1, 0, abort_flag, nullptr, 0);
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
@@ -314,7 +310,6 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   ph_s ^= 1;
   tc_fence_after();
   if (tid == 0 && has_next && PC == 0) issue_q(next_tile);   // no child logits will read this Q tile
-  if (tid == 0 && early_s) issue_vp(tile);              // S is done and so is the last value MMA of the tile before
   // This thread's QW (<= 64) parent logits are read from TMEM once and stay in registers through the
   // maximum, the exponentials, the importance sums and the conversion to bf16.
   float a[QW];
@@ -612,8 +607,6 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     mbar_wait(bar_pv, ph_pv, abort_flag, p.status_word, DEV_TIMEOUT_ATTEND);
     ph_pv ^= 1;
     tc_fence_after();
-    // the parents' value MMA is done: the upper halves of the weight tile and of the value tile are free
-    if (tid == 0 && early_s && has_next && e0 == 0) issue_cp(next_tile);
     // value rows of this chunk (the same gather as for its codeword rows).  Asynchronous copies: they land
     // while the chunk's logits are turned into weights.  Padding rows are zero: they meet finite weights.
     gather_rows(Vs, Vch, e0);
@@ -710,9 +703,6 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     umma_desc_sw128(ca + (k / 4) * np16 * 128 + (k % 4) * 32), idesc, k > 0);
         umma_commit(bar_s);
       }
-    } else if (tid == kScLane && early_s && has_next) {
-      // every thread has read the last child logits (barrier above): the next tile's parent logits
-      issue_s(tmem_base, ph_in ^ 1);
     }
   }
 
@@ -722,7 +712,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tc_fence_after();
   // the last value MMA has released the weight tile and the value tile: the next tile's codebook and
   // parent value rows load while this tile's output is written
-  if (tid == 0 && has_next && !early_s) {
+  if (tid == 0 && has_next) {
     issue_cp(next_tile);
     if (kStageInCC) issue_vp(next_tile);
   }
