@@ -443,16 +443,22 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint32_t kj = keys[j];
         const int span = M / kT, kb = part * span;
         int g0 = 0, g1 = 0, g2 = 0, g3 = 0;              // four independent counters: no serial add chain
-#pragma unroll 4
-        for (int k = kb; k < kb + span; k += 4) {
-          const uint4 kk = *reinterpret_cast<const uint4*>(keys + k);
-          asm("{\n\t.reg .pred p0, p1, p2, p3;\n\t"
-              "setp.gt.u32 p0, %4, %8;\n\tsetp.gt.u32 p1, %5, %8;\n\t"
-              "setp.gt.u32 p2, %6, %8;\n\tsetp.gt.u32 p3, %7, %8;\n\t"
-              "@p0 add.s32 %0, %0, 1;\n\t@p1 add.s32 %1, %1, 1;\n\t"
-              "@p2 add.s32 %2, %2, 1;\n\t@p3 add.s32 %3, %3, 1;\n\t}"
-              : "+r"(g0), "+r"(g1), "+r"(g2), "+r"(g3)
-              : "r"(kk.x), "r"(kk.y), "r"(kk.z), "r"(kk.w), "r"(kj));
+        // 16 keys per trip (span is a multiple of 16): the four 16-byte loads are in flight together
+        // instead of one load -> compare -> add chain per trip
+        for (int k = kb; k < kb + span; k += 16) {
+          uint4 kq[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) kq[u] = *reinterpret_cast<const uint4*>(keys + k + 4 * u);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            asm("{\n\t.reg .pred p0, p1, p2, p3;\n\t"
+                "setp.gt.u32 p0, %4, %8;\n\tsetp.gt.u32 p1, %5, %8;\n\t"
+                "setp.gt.u32 p2, %6, %8;\n\tsetp.gt.u32 p3, %7, %8;\n\t"
+                "@p0 add.s32 %0, %0, 1;\n\t@p1 add.s32 %1, %1, 1;\n\t"
+                "@p2 add.s32 %2, %2, 1;\n\t@p3 add.s32 %3, %3, 1;\n\t}"
+                : "+r"(g0), "+r"(g1), "+r"(g2), "+r"(g3)
+                : "r"(kq[u].x), "r"(kq[u].y), "r"(kq[u].z), "r"(kq[u].w), "r"(kj));
+          }
         }
         gt = (g0 + g1) + (g2 + g3);
       }
@@ -560,11 +566,21 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     // (all of it under the default rule, the share of the keys that moved to children under PARENT_STAYS);
     // the row's NQ threads split the P look-ups
     float fix = 0.f;
-    for (int u = cq; u < min(P, M); u += NQ) {
-      const int j = sel_list[u];
-      const uint16_t hv =
-          *reinterpret_cast<const uint16_t*>(CA + (j >> 6) * (kRows * 128) + sw128_offset(r, j & 63));
-      fix = fmaf(__uint_as_float((uint32_t)hv << 16), 1.f - cntk[j], fix);
+    const int nsel = min(P, M);
+    for (int u0 = cq; u0 < nsel; u0 += 4 * NQ) {         // four look-ups in flight per trip
+      int jj[4];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) jj[t] = sel_list[min(u0 + t * NQ, nsel - 1)];
+      float wv[4], kv[4];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const uint16_t hv =
+            *reinterpret_cast<const uint16_t*>(CA + (jj[t] >> 6) * (kRows * 128) + sw128_offset(r, jj[t] & 63));
+        wv[t] = __uint_as_float((uint32_t)hv << 16);
+        kv[t] = (u0 + t * NQ < nsel) ? 1.f - cntk[jj[t]] : 0.f;
+      }
+#pragma unroll
+      for (int t = 0; t < 4; ++t) fix = fmaf(wv[t], kv[t], fix);
     }
     xz2[cq * kRows + r] = zall - fix;
   }
