@@ -47,7 +47,7 @@ MAX_REPEATS = 200
 L2_POLICY = "inputs rotate through independent copies whose total footprint exceeds twice the L2"
 # Datasheet figures (HGX B200: HBM3e 7.7 TB/s, dense bf16 2.25 PFLOP/s), printed beside the measured peaks.
 NOMINAL = dict(hbm_gbs=7700.0, tflops=2250.0)
-KERNELS_PER_STEP = 4          # assign, leaf scatter, finalize, attend
+KERNELS_PER_STEP = 5          # codeword norms, assign, leaf scatter, finalize, attend
 
 
 def parse_workload(name: str):

@@ -41,9 +41,12 @@
  *
  * Errors: every entry point validates its arguments on the host and returns a status
  * without launching anything when they are unusable.  Shapes outside the supported
- * envelope give AVQ_ERR_UNSUPPORTED; there is no silent fallback.  Device-side waits are
- * bounded; a kernel that gives up records a code in the workspace header which
- * avq_check() reports as AVQ_ERR_DEVICE_TIMEOUT.
+ * envelope give AVQ_ERR_UNSUPPORTED; there is no silent fallback.  Device-side waits on
+ * barriers (loads, tensor-core completion) are bounded; a kernel that gives up records a
+ * code in the workspace header which avq_check() reports as AVQ_ERR_DEVICE_TIMEOUT.  Two
+ * hardware waits carry no limit of their own and end when the work ahead of them on the
+ * GPU ends: the allocation of tensor memory by a thread block and the dependency wait
+ * between the kernels of one call.
  */
 #ifndef AVQ_ATTN_H_
 #define AVQ_ATTN_H_

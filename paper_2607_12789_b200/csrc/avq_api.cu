@@ -73,6 +73,7 @@ Layout make_layout(const avq_problem& p, int32_t /*P*/, int32_t /*block_q*/) {
       L.Vsb = take(2 * BH * p.M * p.d);
       L.rho = take(sizeof(float) * BH * p.M);
     }
+    L.cnorm = take(sizeof(float) * (size_t)p.H * p.M);
   }
   L.total = off;
   return L;
@@ -112,7 +113,7 @@ avq_status avq_assign(const avq_problem* prob, const void* K, const void* Cp, co
   if (!aligned16(K) || !aligned16(Cp) || !aligned16(Cc) || !aligned16(parent_idx) || !aligned16(child_idx))
     return AVQ_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (use_tensor_path(*prob)) return tc_assign(*prob, K, Cp, Cc, parent_idx, child_idx, nullptr, nullptr, 0, st);
+  if (use_tensor_path(*prob)) return tc_assign(*prob, K, Cp, Cc, parent_idx, child_idx, nullptr, nullptr, 0, nullptr, st);
   return simt_assign(*prob, K, Cp, Cc, parent_idx, child_idx, st);
 }
 
@@ -137,6 +138,7 @@ struct Regions {
   float *Vp, *np_, *Vc, *nc;
   void *Vpb, *Vcb, *Vsb;
   float* rho;
+  float* cnorm;
 };
 Regions carve(void* workspace, const Layout& L) {
   char* ws = static_cast<char*>(workspace);
@@ -152,6 +154,7 @@ Regions carve(void* workspace, const Layout& L) {
   r.Vcb = ws + L.Vcb;
   r.Vsb = L.Vsb ? ws + L.Vsb : nullptr;
   r.rho = L.rho ? reinterpret_cast<float*>(ws + L.rho) : nullptr;
+  r.cnorm = L.cnorm ? reinterpret_cast<float*>(ws + L.cnorm) : nullptr;
   return r;
 }
 avq_status attend_stage(const avq_problem& p, const Regions& r, const void* Q, const void* Cp, const void* Cc,
@@ -190,7 +193,10 @@ avq_status avq_forward(const avq_problem* prob, const void* Q, const void* K, co
   const Regions r = carve(workspace, L);
   if (use_tensor_path(p)) {
     // status header, leaf sums and leaf counts are adjacent: the assign grid clears them on the side
-    s = tc_assign(p, K, Cp, Cc, r.pidx, r.cidx, r.status_word, workspace, L.zero_end, st);
+    // The codeword norms as a pass of their own pay once many CTAs share them and a codebook is large: measured
+    // c3 (128 CTAs per head, M d = 32768) -4 us, c2 (M d = 8192) +-0, c1 +1.4 us (the extra launch).
+    const bool norms_pass = (size_t)p.M * p.d >= 16384 && (size_t)p.B * p.H * ((p.Nk + 127) / 128) >= 592;
+    s = tc_assign(p, K, Cp, Cc, r.pidx, r.cidx, r.status_word, workspace, L.zero_end, norms_pass ? r.cnorm : nullptr, st);
     if (s != AVQ_OK) return s;
     s = tc_aggregate(p, V, r.pidx, r.cidx, r.Vp, r.np_, r.Vc, r.nc, r.Vpb, r.Vcb, r.Vsb, r.rho, true, r.status_word, st);
   } else {

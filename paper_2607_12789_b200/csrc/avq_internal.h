@@ -23,6 +23,7 @@ struct Layout {
   size_t Vcb = 0;          // bf16 [B,H,M,C,d]    copy of Vc (tensor-core path only)
   size_t Vsb = 0;          // bf16 [B,H,M,d]      stay residual rows (tensor-core path, PARENT_STAYS)
   size_t rho = 0;          // f32 [B,H,M]         share of a parent's keys that stay
+  size_t cnorm = 0;        // f32 [H,M]           squared norms of the parent codewords (tensor-core path)
   size_t total = 0;
 };
 
@@ -57,9 +58,11 @@ constexpr size_t kSimtAttendSmemLimit = 200 * 1024;
 
 // ---- tensor-core kernels (avq_tc_*.cu) ----
 // zero_base / zero_bytes: a region (multiple of 16 bytes, or none) the assign grid clears on the side
+// cnorm: scratch for [H, M] squared codeword norms, filled by a small kernel ahead of the assign grid; when
+// null every assign CTA computes the norms of its head itself
 avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const void* Cc,
                      int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, void* zero_base,
-                     size_t zero_bytes, cudaStream_t st);
+                     size_t zero_bytes, float* cnorm, cudaStream_t st);
 avq_status tc_aggregate(const avq_problem& p, const void* V, const int32_t* parent_idx,
                         const int32_t* child_idx, float* Vp, float* np_, float* Vc, float* nc,
                         void* Vpb, void* Vcb, void* Vsb, float* rho, bool pre_zeroed, int32_t* status_word,

@@ -72,6 +72,33 @@ __device__ double exact_dist_smem(const unsigned char* Ks, int row, const __nv_b
   return s;
 }
 
+// ||c||^2 of every parent codeword of every head, once per call: a per-head constant that otherwise each of
+// the Nk / 128 assign CTAs of every (batch, head) recomputes.  Eight lanes per codeword row.
+template <int D>
+__global__ void __launch_bounds__(256) code_norms_kernel(const __nv_bfloat16* __restrict__ Cp, float* __restrict__ cnorm,
+                                                         int rows) {
+  pdl_launch_dependents();   // the assign grid may start its set-up and loads
+  const int row = (blockIdx.x * 256 + threadIdx.x) >> 3, part = threadIdx.x & 7;
+  float s = 0.f;
+  if (row < rows) {
+    const uint4* src = reinterpret_cast<const uint4*>(Cp + (size_t)row * D) + part;
+#pragma unroll
+    for (int t = 0; t < D / 64; ++t) {
+      const uint4 v = __ldg(src + 8 * t);
+      const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        s = fmaf(bf_lo(wv[e]), bf_lo(wv[e]), s);
+        s = fmaf(bf_hi(wv[e]), bf_hi(wv[e]), s);
+      }
+    }
+  }
+  s += __shfl_xor_sync(0xffffffffu, s, 1);
+  s += __shfl_xor_sync(0xffffffffu, s, 2);
+  s += __shfl_xor_sync(0xffffffffu, s, 4);
+  if (row < rows && part == 0) cnorm[row] = s;
+}
+
 // NL = 16-byte loads per lane that cover one parent's C x d block of children: C * d / 256.
 // STAYS: Algorithm 1's masked scatter - a key moves to its nearest child only if that child is strictly
 // closer than the parent (child index -1 otherwise).
@@ -80,7 +107,8 @@ __global__ void __launch_bounds__(kThreadsA, assign_min_ctas(D, NL))
 tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmCp,
                  const __nv_bfloat16* __restrict__ Cp, const __nv_bfloat16* __restrict__ Cc,
                  int32_t* __restrict__ pidx, int32_t* __restrict__ cidx, int H, int Nk, int M, int C,
-                 uint32_t tmem_cols, int32_t* status_word, uint4* __restrict__ zero_base, uint32_t zero_units) {
+                 uint32_t tmem_cols, int32_t* status_word, uint4* __restrict__ zero_base, uint32_t zero_units,
+                 const float* cnorm_g) {
   // 1024-byte alignment (swizzle atoms) is requested from the launch, not computed from the pointer, so
   // that the compiler keeps every access in the shared address space.
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -129,6 +157,9 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       tma_load_2d(Cs + s * M * 128, &tmCp, s * 64, h * M, &bars[0]);
     }
   }
+  // tcgen05.alloc blocks while the SM's columns are taken (four CTAs of 256 columns share an SM at d = 64,
+  // M > 128: two run, two wait here).  The holders need nothing from the waiters and free their columns
+  // before they end, so the wait is finite; it is the one device-side wait without a time limit of its own.
   if (warp == 1) {                                   // not the warp whose lane 0 is busy issuing the loads
     tmem_alloc(tmem_slot, tmem_cols);
     tmem_relinquish();
@@ -150,7 +181,16 @@ tc_assign_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     umma_commit(&bars[1]);
   }
 
-  // ||c_m||^2 from the staged codebook (and its maximum), half of ||k||^2 per thread
+  // ||c_m||^2 (and its maximum): from the array the kernel ahead of this one filled, or from the staged
+  // codebook; half of ||k||^2 per thread
+  if (cnorm_g) {
+    pdl_wait();
+    for (int m = tid; m < M; m += kThreadsA) {
+      const float s = ld_after_wait(cnorm_g + (size_t)h * M + m);
+      cnorm[m] = s;
+      atomicMax(cmax_bits, __float_as_uint(s));
+    }
+  } else
   for (int m = tid; m < M; m += kThreadsA) {
     float s = 0.f;
 #pragma unroll
@@ -363,7 +403,7 @@ uint32_t pow2_cols(int n) {
 
 template <int D, int NL, bool STAYS>
 avq_status launch(const avq_problem& p, const void* K, const void* Cp, const void* Cc, int32_t* pidx,
-                  int32_t* cidx, int32_t* status_word, void* zero_base, size_t zero_bytes, cudaStream_t st) {
+                  int32_t* cidx, int32_t* status_word, void* zero_base, size_t zero_bytes, float* cnorm, cudaStream_t st) {
   CUtensorMap tmK, tmCp;
   const uint64_t BH = (uint64_t)p.B * p.H;
   {
@@ -392,23 +432,28 @@ avq_status launch(const avq_problem& p, const void* K, const void* Cp, const voi
     if (dev >= 0 && dev < 64) configured[dev] = smem;
   }
   dim3 grid((p.Nk + kKeys - 1) / kKeys, (unsigned)BH);
-  kern<<<grid, kThreadsA, smem, st>>>(tmK, tmCp, static_cast<const __nv_bfloat16*>(Cp),
-                                      static_cast<const __nv_bfloat16*>(Cc), pidx, cidx, p.H, p.Nk, p.M, p.C,
-                                      pow2_cols(p.M), status_word, static_cast<uint4*>(zero_base),
-                                      (uint32_t)(zero_bytes / 16));
-  return cuda_ok(cudaGetLastError());
+  if (cnorm) {
+    const int rows = p.H * p.M;
+    code_norms_kernel<D><<<(rows * 8 + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(Cp), cnorm, rows);
+    if (cudaGetLastError() != cudaSuccess) return AVQ_ERR_CUDA;
+  }
+  // launched as a dependent of the norms kernel when there is one: set-up, loads and the MMA overlap it
+  return cuda_ok(launch_pdl(kern, grid, dim3(kThreadsA), smem, st, cnorm != nullptr, tmK, tmCp,
+                            static_cast<const __nv_bfloat16*>(Cp), static_cast<const __nv_bfloat16*>(Cc), pidx, cidx,
+                            p.H, p.Nk, p.M, p.C, pow2_cols(p.M), status_word, static_cast<uint4*>(zero_base),
+                            (uint32_t)(zero_bytes / 16), static_cast<const float*>(cnorm)));
 }
 
 }  // namespace
 
 avq_status tc_assign(const avq_problem& p, const void* K, const void* Cp, const void* Cc,
                      int32_t* parent_idx, int32_t* child_idx, int32_t* status_word, void* zero_base,
-                     size_t zero_bytes, cudaStream_t st) {
+                     size_t zero_bytes, float* cnorm, cudaStream_t st) {
   if (zero_bytes % 16 != 0 || (zero_bytes / 16) >> 31) return AVQ_ERR_WORKSPACE;
   const bool stays = (p.flags & AVQ_FLAG_PARENT_STAYS) != 0;
 #define AVQ_ASSIGN(DD, NN)                                                                                     \
-  (stays ? launch<DD, NN, true>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st) \
-         : launch<DD, NN, false>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, st))
+  (stays ? launch<DD, NN, true>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, cnorm, st) \
+         : launch<DD, NN, false>(p, K, Cp, Cc, parent_idx, child_idx, status_word, zero_base, zero_bytes, cnorm, st))
   if (p.d == 64) return p.C == 4 ? AVQ_ASSIGN(64, 1) : AVQ_ASSIGN(64, 2);
   return p.C == 4 ? AVQ_ASSIGN(128, 2) : AVQ_ASSIGN(128, 4);
 #undef AVQ_ASSIGN

@@ -227,6 +227,10 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     issue_q(blockIdx.x);
     issue_cp(blockIdx.x);
   }
+  // TMEM is allocated before the dependency wait.  tcgen05.alloc blocks until the columns are free and the
+  // wait returns only when the kernels before this one have finished; neither can hold the other up: the
+  // columns an earlier kernel's CTAs own are released when those CTAs end, which needs nothing from this
+  // kernel, and CTAs of this kernel release theirs on every path (including the early exit below).
   if (warp == 1) {                                   // not the warp whose lane 0 is busy issuing the loads
     tmem_alloc(tmem_slot, p.tmem_cols);
     tmem_relinquish();
