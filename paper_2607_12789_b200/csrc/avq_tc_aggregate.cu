@@ -126,12 +126,24 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
 
   // ---- leaf of every key and its rank among the chunk's keys of that leaf
   uint32_t lr[kSortKeysPerThread];                     // leaf << 16 | rank
+  // all index loads first: they are ordered statements (behind the dependency wait) that the compiler will
+  // not move across the shared-memory atomics below, so issued one key at a time each would cost a round trip
+  int av[kSortKeysPerThread], cv[kSortKeysPerThread];
+#pragma unroll
+  for (int t = 0; t < kSortKeysPerThread; ++t) {
+    const int j = tid + t * kSortThreads;
+    av[t] = cv[t] = 0;
+    if (j < n) {
+      av[t] = tc::ld_after_wait(pidx + kb + j);
+      cv[t] = tc::ld_after_wait(cidx + kb + j);
+    }
+  }
 #pragma unroll
   for (int t = 0; t < kSortKeysPerThread; ++t) {
     const int j = tid + t * kSortThreads;
     lr[t] = 0xFFFFFFFFu;
     if (j < n) {
-      const int a = tc::ld_after_wait(pidx + kb + j), c = tc::ld_after_wait(cidx + kb + j);   // behind the wait
+      const int a = av[t], c = cv[t];
       if (a < 0 || a >= M || c < -1 || c >= C) {       // caller-supplied index out of range: skip the key, flag it
         if (status_word) atomicCAS(status_word, 0, DEV_BAD_INDEX);
       } else {
@@ -232,6 +244,16 @@ leaf_sorted_kernel(const __nv_bfloat16* __restrict__ V, const int32_t* __restric
 
 // One CTA: kPer consecutive parents of one (batch, head) (8 with four children each, 4 with eight: 32 leaf
 // rows); thread k owns head-dimension index k.  Every load is issued before the first use.
+// 1 / n for a key count (a small positive integer held in a float): the approximate reciprocal (one XU
+// instruction, within an ulp or two) is far inside what the bf16 rounding of the mean leaves of it.  The
+// correctly rounded __frcp_rn is a long dependent sequence, 40 of which per thread were most of this kernel's
+// time on the few warps it runs with.
+__device__ __forceinline__ float fast_rcp(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 template <int D, int C>
 __global__ void __launch_bounds__(D)
 finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, float* __restrict__ Vp,
@@ -266,11 +288,11 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
       s += x[mm][c];
       n += cn[mm][c];
       // the attention kernel takes per-codeword MEANS: the count rides in its softmax weights
-      if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(cn[mm][c] > 0.f ? x[mm][c] * __frcp_rn(cn[mm][c]) : 0.f);
+      if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(cn[mm][c] > 0.f ? x[mm][c] * fast_rcp(cn[mm][c]) : 0.f);
     }
     ntot[mm] = n;
     Vp[row * D + k] = s;
-    const float rn = n > 0.f ? __frcp_rn(n) : 0.f;
+    const float rn = n > 0.f ? fast_rcp(n) : 0.f;
     if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(s * rn);
     // what a refined parent keeps under the PARENT_STAYS rule, per key of the parent: its weight in the
     // attention kernel is A n_p, so the row is Vbar_stay / n_p and the count n_stay / n_p

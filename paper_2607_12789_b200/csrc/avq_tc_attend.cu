@@ -90,10 +90,13 @@ __device__ __forceinline__ void row_sync(int q) {
 
 // Multiplies 16 fp32 weights by their codewords' key counts, rounds the products to bf16, stores them at
 // (row r, columns col0..col0+15) of the K-major swizzled A tile, and returns the sum of the rounded
-// products (the denominator is built from exactly what the value MMA multiplies).
+// products (the denominator is built from exactly what the value MMA multiplies).  KEEP: each product
+// enters that sum times keep16[] (the share of its own term a parent keeps once it is refined).
+template <bool KEEP>
 __device__ __forceinline__ float store_weights16(unsigned char* A, int r, int col0, const float* cnt16,
-                                                 const float (&a)[16]) {
+                                                 const float* keep16, const float (&a)[16]) {
   const float4* n4 = reinterpret_cast<const float4*>(cnt16);
+  const float4* k4 = reinterpret_cast<const float4*>(keep16);
   uint32_t pk[8];
   float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;         // independent partial sums: no 16-deep add chain
 #pragma unroll
@@ -101,10 +104,18 @@ __device__ __forceinline__ float store_weights16(unsigned char* A, int r, int co
     const float4 n = n4[u];
     const uint32_t p0 = pack_bf16(a[4 * u] * n.x, a[4 * u + 1] * n.y);
     const uint32_t p1 = pack_bf16(a[4 * u + 2] * n.z, a[4 * u + 3] * n.w);
-    z0 += __uint_as_float(p0 << 16);
-    z1 += __uint_as_float(p0 & 0xFFFF0000u);
-    z2 += __uint_as_float(p1 << 16);
-    z3 += __uint_as_float(p1 & 0xFFFF0000u);
+    if constexpr (KEEP) {
+      const float4 k = k4[u];
+      z0 = fmaf(__uint_as_float(p0 << 16), k.x, z0);
+      z1 = fmaf(__uint_as_float(p0 & 0xFFFF0000u), k.y, z1);
+      z2 = fmaf(__uint_as_float(p1 << 16), k.z, z2);
+      z3 = fmaf(__uint_as_float(p1 & 0xFFFF0000u), k.w, z3);
+    } else {
+      z0 += __uint_as_float(p0 << 16);
+      z1 += __uint_as_float(p0 & 0xFFFF0000u);
+      z2 += __uint_as_float(p1 << 16);
+      z3 += __uint_as_float(p1 & 0xFFFF0000u);
+    }
     pk[2 * u] = p0;
     pk[2 * u + 1] = p1;
   }
@@ -119,7 +130,8 @@ __device__ __forceinline__ float store_weights16(unsigned char* A, int r, int co
 // overlap each other's load / MMA / softmax phases; the largest take NQ = 4.
 // CT = parent tile width (64, 128 or 256, >= M), a compile-time constant so that every shared-memory
 // offset folds into the instruction stream instead of occupying a register.
-template <int D, int NQ, int CT>
+// FUSE = the weight conversion runs inside the exponential loop (chosen by the launcher from CT, P and M).
+template <int D, int NQ, int CT, bool FUSE>
 __global__ void __launch_bounds__(128 * NQ, 4 / NQ)
 tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmCp,
                  const __grid_constant__ CUtensorMap tmVpb, const __grid_constant__ CUtensorMap tmY,
@@ -174,6 +186,10 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // buffer, which are adjacent and together as large (the next tile's value rows then load a little later).
   constexpr bool kChain = true;
   constexpr bool kStageInCC = CT >= 128;
+  // weight conversion inside the exponential loop (see there): pays where few CTAs share the SM and P is small
+  // against M; measured slower for the 64-column tiles (four CTAs per SM already fill each other's gaps) and
+  // for P near M (the P look-ups per row cost more than the overlap gains)
+  constexpr bool fuse = FUSE;
   auto issue_q = [&](int t) {                            // thread 0 only
     const int tb = t / p.nblk, ti0 = (t - tb * p.nblk) * kRows;
     mbar_expect_tx(bar_q, (uint32_t)(kSubD * kRows * 128));
@@ -371,13 +387,16 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           zf2 = fmaf(a[c0 + 4 * u + 2], n.z, zf2);
           zf3 = fmaf(a[c0 + 4 * u + 3], n.w, zf3);
         }
-        // The bf16 weights go to shared memory (over the dead codebook) right here: the exponentials keep the
-        // XU pipe busy and the conversion (ALU pipe, stores) fills the issue slots they leave empty.  The
-        // selection is not known yet; what it removes is taken out of the denominator afterwards.
-        float am[16];
+        // Large tiles with few parents to refine: the bf16 weights go to shared memory (over the dead
+        // codebook) right here - the exponentials keep the XU pipe busy and the conversion (ALU pipe, stores)
+        // fills the issue slots they leave empty.  The selection is not known yet; what it removes is taken
+        // out of the denominator afterwards (P look-ups per row).
+        if constexpr (fuse) {
+          float am[16];
 #pragma unroll
-        for (int e = 0; e < 16; ++e) am[e] = a[c0 + e];
-        zall += store_weights16(CA, r, colbase + c0, cnt + colbase + c0, am);
+          for (int e = 0; e < 16; ++e) am[e] = a[c0 + e];
+          zall += store_weights16<false>(CA, r, colbase + c0, cnt + colbase + c0, nullptr, am);
+        }
       }
     }
     zfull = (zf0 + zf1) + (zf2 + zf3);
@@ -565,7 +584,21 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (p.Vsb) stay = __ldg(reinterpret_cast<const uint4*>(p.Vsb + ((size_t)bh * M + row) * D) + ch);
     *reinterpret_cast<uint4*>(Vs + (ch >> 3) * (M * 128) + sw128_offset(row, (ch & 7) * 8)) = stay;
   }
-  {
+  if constexpr (!fuse) {
+    // bf16 weights into shared memory (over the dead codebook) + their denominator; a refined parent's
+    // rounded weight enters the denominator with the share of its own term that it keeps (cntk)
+    float zloc = 0.f;
+#pragma unroll
+    for (int c0 = 0; c0 < QW; c0 += 16) {
+      if (c0 < my_cols) {
+        float am[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) am[e] = a[c0 + e];
+        zloc += store_weights16<true>(CA, r, colbase + c0, cnt + colbase + c0, cntk + colbase + c0, am);
+      }
+    }
+    xz2[cq * kRows + r] = zloc;
+  } else {
     // denominator of the parent pass from the rounded weights, less what the refined parents no longer carry
     // (all of it under the default rule, the share of the keys that moved to children under PARENT_STAYS);
     // the row's NQ threads split the P look-ups
@@ -684,7 +717,7 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         tmem_ld16(t_sc + c0, a);
 #pragma unroll
         for (int e = 0; e < 16; ++e) a[e] = ex2(fminf(fmaf(a[e], sc, negm), kLazyLog2));   // clamp: empty children
-        zloc += store_weights16(CA, r, cq * QWC + c0, cntc + cq * QWC + c0, a);
+        zloc += store_weights16<false>(CA, r, cq * QWC + c0, cntc + cq * QWC + c0, nullptr, a);
       }
       xz2[cq * kRows + r] = zloc;
     }
@@ -777,11 +810,11 @@ size_t attend_smem(int D, int CT, int CHW, int NQ, int MC) {
   return b + 64 + sizeof(float) * (size_t)MC;
 }
 
-template <int D, int NQ, int CT>
-avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUtensorMap& tmVpb,
+template <int D, int NQ, int CT, bool FUSE>
+avq_status launch_nq_f(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUtensorMap& tmVpb,
                      const CUtensorMap& tmY, const AttendParams& a, unsigned BH, size_t smem, bool chained,
                      cudaStream_t st) {
-  auto kern = tc_attend_kernel<D, NQ, CT>;
+  auto kern = tc_attend_kernel<D, NQ, CT, FUSE>;
   // The limit is set once per device and instantiation (setting it again is harmless if two threads race).
   static size_t configured[64] = {};
   int dev = 0;
@@ -805,6 +838,19 @@ avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUte
   // and Q was complete before the call, so the attention kernel may start as its programmatic dependent.
   // A stand-alone avq_attend is launched plainly: the work before it in the stream may be producing Q.
   return cuda_ok(launch_pdl(kern, grid, dim3(128 * NQ), smem, st, chained, tmQ, tmCp, tmVpb, tmY, a));
+}
+
+template <int D, int NQ, int CT>
+avq_status launch_nq(const CUtensorMap& tmQ, const CUtensorMap& tmCp, const CUtensorMap& tmVpb,
+                     const CUtensorMap& tmY, const AttendParams& a, unsigned BH, size_t smem, bool chained,
+                     cudaStream_t st) {
+  // conversion inside the exponential loop: measured to pay for the larger tiles when P is small against M
+  // (c2 45.1 -> 43.3 us, c3 188 -> 184 us) and to cost for 64-column tiles (N=16384 M=64 P=16: 43 -> 47 us)
+  // and for P near M (N=65536 M=128 P=128: 615 -> 649 us)
+  if constexpr (CT >= 128) {
+    if (4 * a.P <= a.M) return launch_nq_f<D, NQ, CT, true>(tmQ, tmCp, tmVpb, tmY, a, BH, smem, chained, st);
+  }
+  return launch_nq_f<D, NQ, CT, false>(tmQ, tmCp, tmVpb, tmY, a, BH, smem, chained, st);
 }
 
 template <int D>
