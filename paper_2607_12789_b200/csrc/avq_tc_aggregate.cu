@@ -255,55 +255,46 @@ __device__ __forceinline__ float fast_rcp(float x) {
 }
 
 template <int D, int C>
-__global__ void __launch_bounds__(D)
+__global__ void __launch_bounds__(D * ((C == 4) ? 8 : 4))
 finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, float* __restrict__ Vp,
                 float* __restrict__ np_, __nv_bfloat16* __restrict__ Vpb, __nv_bfloat16* __restrict__ Vcb,
                 __nv_bfloat16* __restrict__ Vsb, float* __restrict__ rho, int M) {
+  // One CTA = kPer consecutive parents of one (batch, head); thread (k, mm) owns head-dimension index k of
+  // parent mm: C + 1 row loads, C + 2 counts, a handful of stores.  The kernel is a load round trip followed
+  // by a little arithmetic, so it wants many short threads, not few long ones.
   constexpr int kPer = (C == 4) ? 8 : 4;
   tc::pdl_launch_dependents();
   tc::pdl_wait();                                    // the leaf sums come from the kernel before
-  const int bh = blockIdx.y, m0 = blockIdx.x * kPer, k = threadIdx.x;
-  float x[kPer][C], cn[kPer][C], stay[kPer], nstay[kPer];
+  const int bh = blockIdx.y, k = threadIdx.x, mm = threadIdx.y;
+  const size_t row = (size_t)bh * M + blockIdx.x * kPer + mm;
+  // Everything read here is written by the kernel before this one: the loads are statements the compiler
+  // cannot move ahead of the dependency wait above (an ordinary load of np_ was seen to be scheduled ahead of
+  // it, reading counts the scatter had not finished).
+  float x[C], cn[C];
 #pragma unroll
-  for (int mm = 0; mm < kPer; ++mm) {
-    const size_t row = (size_t)bh * M + m0 + mm;
-#pragma unroll
-    for (int c = 0; c < C; ++c) {
-      x[mm][c] = tc::ld_after_wait(Vc + (row * C + c) * D + k);
-      cn[mm][c] = tc::ld_after_wait(nc + row * C + c);
-    }
-    // Everything read here is written by the kernel before this one: the loads are statements the compiler
-    // cannot move ahead of the dependency wait above (an ordinary load of np_ was seen to be scheduled ahead
-    // of it, reading counts the scatter had not finished).
-    stay[mm] = tc::ld_after_wait(Vp + row * D + k);   // zero unless keys stay
-    nstay[mm] = tc::ld_after_wait(np_ + row);         // keys that stay
+  for (int c = 0; c < C; ++c) {
+    x[c] = tc::ld_after_wait(Vc + (row * C + c) * D + k);
+    cn[c] = tc::ld_after_wait(nc + row * C + c);
   }
-  float ntot[kPer];
+  const float stay = tc::ld_after_wait(Vp + row * D + k);   // zero unless keys stay
+  const float nstay = tc::ld_after_wait(np_ + row);         // keys that stay
+  float s = stay, n = nstay;
 #pragma unroll
-  for (int mm = 0; mm < kPer; ++mm) {
-    const size_t row = (size_t)bh * M + m0 + mm;
-    float s = stay[mm], n = nstay[mm];
-#pragma unroll
-    for (int c = 0; c < C; ++c) {
-      s += x[mm][c];
-      n += cn[mm][c];
-      // the attention kernel takes per-codeword MEANS: the count rides in its softmax weights
-      if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(cn[mm][c] > 0.f ? x[mm][c] * fast_rcp(cn[mm][c]) : 0.f);
-    }
-    ntot[mm] = n;
-    Vp[row * D + k] = s;
-    const float rn = n > 0.f ? fast_rcp(n) : 0.f;
-    if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(s * rn);
-    // what a refined parent keeps under the PARENT_STAYS rule, per key of the parent: its weight in the
-    // attention kernel is A n_p, so the row is Vbar_stay / n_p and the count n_stay / n_p
-    if (Vsb) Vsb[row * D + k] = __float2bfloat16_rn(stay[mm] * rn);
-    if (rho && k == 0) rho[row] = nstay[mm] * rn;
+  for (int c = 0; c < C; ++c) {
+    s += x[c];
+    n += cn[c];
+    // the attention kernel takes per-codeword MEANS: the count rides in its softmax weights
+    if (Vcb) Vcb[(row * C + c) * D + k] = __float2bfloat16_rn(cn[c] > 0.f ? x[c] * fast_rcp(cn[c]) : 0.f);
   }
-  __syncthreads();                                     // every thread has read the stay counts
-  if (k == 0) {
-#pragma unroll
-    for (int mm = 0; mm < kPer; ++mm) np_[(size_t)bh * M + m0 + mm] = ntot[mm];
-  }
+  Vp[row * D + k] = s;
+  const float rn = n > 0.f ? fast_rcp(n) : 0.f;
+  if (Vpb) Vpb[row * D + k] = __float2bfloat16_rn(s * rn);
+  // what a refined parent keeps under the PARENT_STAYS rule, per key of the parent: its weight in the
+  // attention kernel is A n_p, so the row is Vbar_stay / n_p and the count n_stay / n_p
+  if (Vsb) Vsb[row * D + k] = __float2bfloat16_rn(stay * rn);
+  if (rho && k == 0) rho[row] = nstay * rn;
+  __syncthreads();                                     // every thread has read its parent's stay count
+  if (k == 0) np_[row] = n;
 }
 
 template <int D, int C>
@@ -363,7 +354,7 @@ avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const i
       return AVQ_ERR_CUDA;
   }
   dim3 g2(p.M / (C == 4 ? 8 : 4), BH);
-  return cuda_ok(tc::launch_pdl(finalize_kernel<D, C>, g2, dim3(D), 0, st, true, static_cast<const float*>(Vc),
+  return cuda_ok(tc::launch_pdl(finalize_kernel<D, C>, g2, dim3(D, C == 4 ? 8 : 4), 0, st, true, static_cast<const float*>(Vc),
                                 static_cast<const float*>(nc), Vp, np_, static_cast<__nv_bfloat16*>(Vpb),
                                 static_cast<__nv_bfloat16*>(Vcb), static_cast<__nv_bfloat16*>(Vsb), rho, p.M));
 }
