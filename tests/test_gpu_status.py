@@ -92,3 +92,33 @@ def test_aggregate_with_caller_indices_stay_keys_and_out_of_range_keys():
             assert np.array_equal(n_c[0, h].cpu().numpy(), rnc)
             assert np.allclose(Vc[0, h].cpu().numpy(), rVc, rtol=2e-5, atol=2e-3)
             assert np.allclose(Vp[0, h].cpu().numpy(), rVp, rtol=2e-5, atol=2e-3)
+
+
+@pytest.mark.parametrize("stays", [False, True])
+def test_back_to_back_forwards_are_repeatable(stays):
+    """The kernels of one call overlap their set-up with the kernel before them (programmatic dependent
+    launch); a load that slipped ahead of the dependency wait would read counts or sums that are not final
+    and show up as a run that differs from the others.  Forty calls back to back (no host synchronisation in
+    between), two shapes: indices, counts and selections identical every time, sums and outputs within the
+    rounding of a different atomic order."""
+    flags = binding.FLAG_PARENT_STAYS if stays else 0
+    for wl in (synth.C1.with_(B=2, H=3, N=1024, seed=61, keys_around_parents=stays),
+               synth.sweep_point(16384, 256, 64).with_(H=1, N=32768, seed=62, keys_around_parents=stays)):   # chained tiles
+        dv = parity.to_device(synth.generate(wl), "bf16")
+        f = binding.Forward(wl.B, wl.H, wl.N, wl.N, wl.d, wl.M, wl.C, wl.P, wl.block_q, dtype=torch.bfloat16,
+                            scale=wl.scale, flags=flags, aux=True)
+        runs = []
+        for _ in range(40):
+            Y = f(dv["Q"], dv["K"], dv["V"], dv["Cp"], dv["Cc"])
+            im = f.intermediates()
+            runs.append((Y.clone(), f.topp.clone(), im["np"].clone(), im["nc"].clone(), im["parent_idx"].clone(),
+                         im["child_idx"].clone(), im["Vp"].clone()))
+        f.check()
+        Y0, t0, np0, nc0, p0, c0, Vp0 = runs[0]
+        assert float(np0.sum()) == wl.B * wl.H * wl.N
+        for Y, t, np_, nc, p, c, Vp in runs[1:]:
+            assert torch.equal(p, p0) and torch.equal(c, c0)
+            assert torch.equal(np_, np0) and torch.equal(nc, nc0)
+            assert torch.equal(t, t0)
+            assert (Vp - Vp0).abs().max().item() <= 1e-3
+            assert (Y.float() - Y0.float()).abs().max().item() <= 2e-2
