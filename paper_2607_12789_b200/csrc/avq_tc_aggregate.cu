@@ -297,16 +297,28 @@ finalize_kernel(const float* __restrict__ Vc, const float* __restrict__ nc, floa
   if (k == 0) np_[row] = n;
 }
 
+// Zeroes the four accumulator arrays of a stand-alone avq_aggregate in one launch (inside avq_forward the
+// assign grid clears them on the side).
+__global__ void __launch_bounds__(256) clear_accumulators_kernel(float* a, size_t na, float* b, size_t nb, float* c,
+                                                                 size_t nc_, float* d, size_t nd) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < na; i += stride) a[i] = 0.f;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nb; i += stride) b[i] = 0.f;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nc_; i += stride) c[i] = 0.f;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nd; i += stride) d[i] = 0.f;
+}
+
 template <int D, int C>
 avq_status run(const avq_problem& p, const void* V, const int32_t* pidx, const int32_t* cidx, float* Vp,
                float* np_, float* Vc, float* nc, void* Vpb, void* Vcb, void* Vsb, float* rho, bool pre_zeroed,
                int32_t* status_word, cudaStream_t st) {
   const unsigned BH = (unsigned)(p.B * p.H);
-  if (!pre_zeroed) {
-    if (cudaMemsetAsync(Vc, 0, sizeof(float) * (size_t)BH * p.M * C * D, st) != cudaSuccess) return AVQ_ERR_CUDA;
-    if (cudaMemsetAsync(nc, 0, sizeof(float) * (size_t)BH * p.M * C, st) != cudaSuccess) return AVQ_ERR_CUDA;
-    if (cudaMemsetAsync(Vp, 0, sizeof(float) * (size_t)BH * p.M * D, st) != cudaSuccess) return AVQ_ERR_CUDA;
-    if (cudaMemsetAsync(np_, 0, sizeof(float) * (size_t)BH * p.M, st) != cudaSuccess) return AVQ_ERR_CUDA;
+  if (!pre_zeroed) {                                   // the stand-alone call: one launch clears the four accumulators
+    const size_t n_c = (size_t)BH * p.M * C, n_p = (size_t)BH * p.M;
+    const size_t total = (n_c + n_p) * (D + 1);
+    const unsigned blocks = (unsigned)((total + 4 * 256 - 1) / (4 * 256) < 2048 ? (total + 4 * 256 - 1) / (4 * 256) : 2048);
+    clear_accumulators_kernel<<<blocks, 256, 0, st>>>(Vc, n_c * D, nc, n_c, Vp, n_p * D, np_, n_p);
+    if (cudaGetLastError() != cudaSuccess) return AVQ_ERR_CUDA;
   }
   // `pre_zeroed` marks the chained call from avq_forward: the kernel before in the stream is the assign
   // kernel, so the scatter may be launched as its programmatic dependent.

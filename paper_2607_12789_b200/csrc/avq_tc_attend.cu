@@ -298,12 +298,12 @@ tc_attend_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // ---- Part 2 reads what the earlier kernels of this call wrote: status word, counts, value sums.
   if (first) {
     pdl_wait();
+    load_counts();                                     // in flight before thread 0 blocks on the status word
     if (tid == 0) {
+      issue_vp(tile);
       // a wait that expired in an earlier CTA or kernel of this call: do not start more work
       early_exit = (p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0);
-      issue_vp(tile);
     }
-    load_counts();
   }
   if (tid < CT) {
     cnt[tid] = n_reg;
