@@ -123,8 +123,10 @@ def test_other_shapes_d128_C8_M96():
 
 
 @pytest.mark.parametrize("wl", [synth.C1.with_(B=2, H=2, N=1500, seed=51), synth.C3.with_(H=2, N=2000, seed=52),
-                                synth.C2.with_(B=1, H=2, N=1100, seed=53)],
-                         ids=["d64_M64_C4", "d128_M256_C4", "d64_M128_C8"])
+                                synth.C2.with_(B=1, H=2, N=1100, seed=53),
+                                synth.sweep_point(4096, 32, 8).with_(H=2, seed=54),      # long head: leaf-ordered aggregate
+                                synth.sweep_point(4096, 128, 128).with_(H=2, seed=55)],  # every parent refined, 4 child chunks
+                         ids=["d64_M64_C4", "d128_M256_C4", "d64_M128_C8", "long_head_M32", "all_refined_M128"])
 def test_parent_stays_on_the_tensor_core_path(wl):
     """Algorithm 1's masked scatter on the tcgen05 path: half of the keys hug their parent and stay with it
     (child index -1), the others move to a child; a refined parent keeps the stay residual."""
